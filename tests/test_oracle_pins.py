@@ -1,0 +1,517 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked against the oracle (no GPU).
+
+Each test cites the passage that fixes the expected value.  A dropped term, a wrong sign or index, or a transposed
+operand anywhere in the oracle should fail at least one of these.
+"""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import (AXIS_COL, AXIS_ROW, GRID_E1M2, GRID_E2M1, GRID_INT4, ROUND_RTNE, ROUND_SR, SCALE_E4M3_TENSOR,
+                    SCALE_FP32, SCALE_POW2)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16_bits(a):
+    """numpy float -> BF16 bit patterns (round to nearest even), via torch's converter."""
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.uint16).numpy().copy()
+
+
+def bf16_vals(bits):
+    return torch.from_numpy(bits.copy()).view(torch.bfloat16).to(torch.float64).numpy()
+
+
+# ------------------------------------------------------------------ Philox (Salmon et al., SC'11 known answers)
+
+def test_philox_known_answers():
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as f:
+        rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 3
+    for w in rows:
+        v = [int(t, 16) for t in w]
+        out = oracle.philox4x32_10(v[0:4], v[4:6])
+        assert out.tolist() == v[6:10]
+
+
+def test_sr_bytes_are_little_endian_bytes_of_the_philox_block():
+    seed, b, variant = 0x1234567890ABCDEF, (5 << 32) | 77, 1
+    words = oracle.philox4x32_10([b & 0xFFFFFFFF, b >> 32, variant, 0x53520000], [seed & 0xFFFFFFFF, seed >> 32])
+    expect = np.frombuffer(words.astype("<u4").tobytes(), dtype=np.uint8)
+    assert oracle.sr_bytes(seed, b, variant).tolist() == expect.tolist()
+
+
+# ------------------------------------------------------------------ Hadamard and RHT (Sec. 2.2)
+
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 16, 32, 64])
+def test_hadamard_is_orthogonal(n):
+    H = oracle.hadamard_matrix(n)
+    tol = 0.0 if n in (1, 4, 16, 64) else 4e-16   # entries are +-2^-k exactly when n is a power of 4
+    assert np.max(np.abs(H.T @ H - np.eye(n))) <= tol
+
+
+def test_hadamard_16_entries_and_sylvester_structure():
+    H = oracle.hadamard_matrix(16)
+    assert set(np.unique(H).tolist()) == {-0.25, 0.25}
+    # Sylvester order: entry (i, j) has sign (-1)^popcount(i & j); first row and column are all positive
+    for i in range(16):
+        for j in range(16):
+            assert H[i, j] == 0.25 * (-1) ** bin(i & j).count("1")
+    H8 = oracle.hadamard_matrix(8)
+    c = 1 / np.sqrt(2.0)
+    assert np.allclose(H, c * np.block([[H8, H8], [H8, -H8]]), atol=1e-16)
+
+
+def test_butterfly_equals_row_vector_times_sign_times_hadamard():
+    H = oracle.hadamard_matrix(16)
+    for mask in (0, 0xFFFF, 0x36A6, 0x0001, 0x8000):
+        eps = np.array([-1.0 if (mask >> i) & 1 else 1.0 for i in range(16)])
+        Hp = np.diag(eps) @ H                      # H' = S H: signs are applied before the Hadamard transform
+        for i in range(16):                        # basis vectors: exact in FP32
+            e = np.zeros(16, dtype=np.float32)
+            e[i] = 1.0
+            assert np.array_equal(oracle.rht16_f32(e, mask).astype(np.float64), Hp[i])
+        rng = np.random.default_rng(mask)
+        x = rng.integers(-64, 64, size=16).astype(np.float32)     # small integers: every FP32 step is exact
+        assert np.array_equal(oracle.rht16_f32(x, mask).astype(np.float64), x.astype(np.float64) @ Hp)
+        x = rng.standard_normal(16).astype(np.float32)
+        assert np.allclose(oracle.rht16_f32(x, mask), x.astype(np.float64) @ Hp, rtol=0, atol=2e-6)
+
+
+def test_rht_is_invertible_and_preserves_the_gemm():
+    rng = np.random.default_rng(3)
+    mask = oracle.rht_sign_mask(1)
+    eps = np.array([-1.0 if (mask >> i) & 1 else 1.0 for i in range(16)])
+    Hp = np.diag(eps) @ oracle.hadamard_matrix(16)
+    assert np.max(np.abs(Hp @ Hp.T - np.eye(16))) == 0.0
+    X = rng.standard_normal((24, 64))
+    W = rng.standard_normal((40, 64))
+    B = np.kron(np.eye(4), Hp)                     # block-diagonal RHT along the shared dimension
+    Y = X @ W.T
+    Yr = (X @ B) @ (W @ B).T
+    assert np.max(np.abs(Y - Yr)) <= 1e-12 * np.max(np.abs(Y))
+    x = rng.standard_normal(16).astype(np.float32)
+    back = oracle.rht16_f32(x, mask).astype(np.float64) @ Hp.T
+    assert np.allclose(back, x, atol=1e-6)
+
+
+def test_sign_mask_depends_on_seed_only_through_philox_word0():
+    for seed in (0, 1, 2, 0xDEADBEEFCAFEF00D):
+        w = oracle.philox4x32_10([0, 0, 0, 0x52485400], [seed & 0xFFFFFFFF, seed >> 32])
+        assert oracle.rht_sign_mask(seed) == int(w[0]) & 0xFFFF
+
+
+# ------------------------------------------------------------------ codebooks and RTNE bins (Sec. 2.1, Sec. 3.1)
+
+def _golden_e2m1():
+    levels, bins = None, []
+    with open(os.path.join(GOLDEN, "e2m1_grid.txt")) as f:
+        for ln in f:
+            w = ln.split()
+            if not w or w[0].startswith("#"):
+                continue
+            if w[0] == "levels":
+                levels = [float(t) for t in w[1:]]
+            elif w[0] == "bin":
+                bins.append([float(t) for t in w[1:]])
+    return levels, bins
+
+
+def test_codebooks():
+    levels, _ = _golden_e2m1()
+    assert oracle.levels(GRID_E2M1).tolist() == levels
+    for grid, gmax in ((GRID_INT4, 7.0), (GRID_E1M2, 1.75)):
+        L = oracle.levels(grid)
+        assert L[0] == 0 and L[-1] == gmax
+        assert np.all(np.diff(L) == L[1])          # equal spacing: l_i = r_i in every bin
+    assert np.array_equal(oracle.levels(GRID_E1M2) * 4, oracle.levels(GRID_INT4))
+
+
+def test_nibble_encodings():
+    # INT4: two's complement; E1M2 / E2M1: sign bit + 3-bit level index.  E1M2 = 1 sign, 1 exponent, 2 mantissa bits
+    # with bias 1: exponent 0 is subnormal (0.mm), exponent 1 is 1.mm.
+    for nib in range(16):
+        q = nib - 16 if nib & 8 else nib
+        assert oracle.nibble_value(GRID_INT4, nib) == q
+        e, mm = (nib >> 2) & 1, nib & 3
+        mag = (mm / 4.0) if e == 0 else (1.0 + mm / 4.0)
+        assert oracle.nibble_value(GRID_E1M2, nib) == (-mag if nib & 8 else mag)
+        ee, m = (nib >> 1) & 3, nib & 1          # E2M1: 2 exponent bits (bias 1), 1 mantissa bit
+        mag = (m * 0.5) if ee == 0 else (1.0 + m * 0.5) * 2.0 ** (ee - 1)
+        assert oracle.nibble_value(GRID_E2M1, nib) == (-mag if nib & 8 else mag)
+
+
+def _exact_rtne(a: Fraction, levels):
+    """Nearest level in exact rational arithmetic; ties to the even index."""
+    best, best_d = 0, abs(a - levels[0])
+    for i in range(1, 8):
+        d = abs(a - levels[i])
+        if d < best_d or (d == best_d and i % 2 == 0):
+            best, best_d = i, d
+    return best
+
+
+@pytest.mark.parametrize("grid", [GRID_INT4, GRID_E1M2, GRID_E2M1])
+def test_rtne_bins_are_midpoint_bins(grid):
+    """Eq. 1: the bin of interior level q_i is ((q_{i-1}+q_i)/2, (q_i+q_{i+1})/2)."""
+    L = oracle.levels(grid)
+    eps = 1e-9
+    for i in range(1, 7):
+        lo, hi = (L[i - 1] + L[i]) / 2, (L[i] + L[i + 1]) / 2
+        for a in (lo + eps, L[i], hi - eps, (lo + hi) / 2):
+            assert oracle.round_rtne(a, grid) == i
+        assert oracle.round_rtne(lo - eps, grid) == i - 1
+        assert oracle.round_rtne(hi + eps, grid) == i + 1
+    assert oracle.round_rtne(0.0, grid) == 0
+    assert oracle.round_rtne(L[7] * 1.5, grid) == 7      # above the grid: saturate
+    # every BF16-representable magnitude in [0, 1.25 g_max], against exact rational arithmetic
+    Lf = [Fraction(float(v)) for v in L]
+    bits = np.arange(0, 0x7F80, dtype=np.uint16)
+    vals = bf16_vals(bits)
+    sel = vals[(vals <= 1.25 * L[7])]
+    step = max(1, sel.size // 6000)
+    for a in sel[::step]:
+        assert oracle.round_rtne(float(a), grid) == _exact_rtne(Fraction(float(a)), Lf)
+
+
+def test_rtne_ties_go_to_even_code():
+    # uniform grid: IEEE round-half-even on the code integer (numpy's rint is the library statement of it)
+    a = np.arange(0, 7.5, 0.125)
+    got = np.array([oracle.round_rtne(float(v), GRID_INT4) for v in a])
+    assert np.array_equal(got, np.rint(a).astype(int))
+    got = np.array([oracle.round_rtne(float(v) / 4, GRID_E1M2) for v in a])
+    assert np.array_equal(got, np.rint(a).astype(int))
+    # E2M1 (1 mantissa bit): ties keep the mantissa bit even, i.e. the even code
+    ties = {0.25: 0.0, 0.75: 1.0, 1.25: 1.0, 1.75: 2.0, 2.5: 2.0, 3.5: 4.0, 5.0: 4.0}
+    L = oracle.levels(GRID_E2M1)
+    for t, expect in ties.items():
+        assert L[oracle.round_rtne(t, GRID_E2M1)] == expect
+
+
+def test_worked_example_bins_of_the_paper():
+    """Footnote to Sec. 3.1: level 2 has bin (1.75, 2.5), l = 0.25, r = 0.5; level 4 the same at double the scale."""
+    _, bins = _golden_e2m1()
+    L = oracle.levels(GRID_E2M1)
+    for level, lo, hi, l_w, r_w, bias in bins:
+        i = L.tolist().index(level)
+        assert (L[i - 1] + L[i]) / 2 == lo and (L[i] + L[i + 1]) / 2 == hi
+        assert (L[i] - L[i - 1]) / 2 == l_w and (L[i + 1] - L[i]) / 2 == r_w
+        assert (l_w - r_w) / 2 == bias
+        t = np.linspace(lo, hi, 200001)[1:-1]
+        got = np.array([L[oracle.round_rtne(float(v), GRID_E2M1)] for v in t[::40]])
+        assert np.all(got == level)
+
+
+@pytest.mark.parametrize("grid", [GRID_INT4, GRID_E1M2, GRID_E2M1])
+def test_per_bin_bias_matches_closed_form(grid):
+    """Eq. 2: E[rho(t) - t | t in B_i] = (2 q_i - q_{i-1} - q_{i+1}) / 4 under locally uniform density."""
+    L = oracle.levels(grid)
+    t = (np.arange(400000) + 0.5) / 400000 * L[7]          # uniform density on (0, g_max)
+    idx = np.array([oracle.round_rtne(float(v), grid) for v in t])
+    for i in range(1, 7):
+        closed = (2 * L[i] - L[i - 1] - L[i + 1]) / 4
+        measured = np.mean(L[idx[idx == i]] - t[idx == i])
+        assert abs(measured - closed) < 2e-4 * L[7]
+    if grid == GRID_E2M1:
+        closed = [(2 * L[i] - L[i - 1] - L[i + 1]) / 4 for i in range(1, 7)]
+        assert closed == [0, 0, 0, -0.125, 0, -0.25]      # the values the paper prints for levels 2 and 4
+    else:
+        assert all((2 * L[i] - L[i - 1] - L[i + 1]) == 0 for i in range(1, 7))
+
+
+def test_bin_bias_through_the_quantizer_pipeline():
+    """Same closed form, measured by orc_bin_bias on the y values the quantizer itself produced (RHT off)."""
+    rng = np.random.default_rng(11)
+    for grid, gmax in ((GRID_INT4, 7.0), (GRID_E2M1, 6.0)):
+        n_blocks = 60000
+        x = rng.uniform(0.0, 1.0, size=(n_blocks, 16)) * rng.choice([-1.0, 1.0], size=(n_blocks, 16))
+        x[:, 0] = 1.0                                     # block amax = 1 exactly -> t = |x| * g_max
+        q = oracle.quantize(bf16_bits(x), AXIS_ROW, rht_block=0, grid=grid, want_y=True)
+        count, mean = oracle.bin_bias(q.y, q.codes, grid)
+        L = oracle.levels(grid)
+        assert count.sum() == n_blocks * 16
+        for i in range(1, 7):
+            closed = (2 * L[i] - L[i - 1] - L[i + 1]) / 4
+            width = (L[i + 1] - L[i - 1]) / 2
+            sigma = width / np.sqrt(12 * count[i])
+            # BF16 input spacing (2^-8 relative) adds a small deterministic lumpiness on top of sampling noise
+            assert abs(mean[i] - closed) < 4 * sigma + 2e-3 * gmax
+
+
+# ------------------------------------------------------------------ stochastic rounding (Sec. 2.1)
+
+@pytest.mark.parametrize("grid", [GRID_INT4, GRID_E1M2, GRID_E2M1])
+def test_sr_probabilities_and_expectation(grid):
+    """Pr[q = g_b] = (a - g_a)/(g_b - g_a): over the 256 equally likely random bytes the count of 'up' outcomes is
+    p*256 rounded to an integer, so E[SR(a)] = a to within half a 1/256 step of the gap."""
+    L = oracle.levels(grid)
+    rng = np.random.default_rng(5)
+    pts = np.concatenate([rng.uniform(0, L[7], 300), L, (L[:-1] + L[1:]) / 2, [L[7] * 1.01, L[7] * 2]])
+    for a in pts:
+        a = float(np.float32(a))
+        out = np.array([oracle.round_sr(a, grid, r) for r in range(256)])
+        if a >= L[7]:
+            assert np.all(out == 7)
+            continue
+        lo = int(np.searchsorted(L, a, side="right") - 1)
+        gap = L[lo + 1] - L[lo]
+        assert set(out.tolist()) <= {lo, lo + 1}
+        p = Fraction(a) - Fraction(float(L[lo]))
+        p = p / Fraction(float(gap))
+        n_up = int(np.sum(out == lo + 1))
+        assert abs(Fraction(n_up, 256) - p) <= Fraction(1, 512)
+        assert abs(np.mean(L[out]) - a) <= gap / 512 + 1e-12
+        # monotone in r: small random bytes round up, large ones round down
+        assert np.all(np.diff((out == lo + 1).astype(int)) <= 0)
+    # exact levels never move
+    for i in range(8):
+        assert all(oracle.round_sr(float(L[i]), grid, r) == i for r in (0, 127, 255))
+
+
+def test_sr_expectation_through_the_quantizer():
+    """E[SR(x)] = x (Sec. 2.1) measured over many Philox-keyed blocks: |mean - x| <= 2^-9 step + 4 sigma."""
+    n_blocks = 40000
+    vals = np.array([1.0, 0.3, -0.55, 0.051, 0.77, -0.123, 0.9, 0.004, -0.31, 0.66, 0.5, -0.999, 0.25, 0.42, -0.8, 0.1])
+    x = np.tile(vals, (n_blocks, 1))
+    bits = bf16_bits(x)
+    xv = bf16_vals(bits)[0]
+    for grid, gmax in ((GRID_INT4, 7.0), (GRID_E2M1, 6.0)):
+        q = oracle.quantize(bits, AXIS_ROW, rht_block=0, grid=grid, rounding=ROUND_SR, seed_sr=2)
+        deq = oracle.dequantize(q)
+        s = float(q.scales[0, 0])
+        assert np.all(q.scales == np.float32(1.0) / np.float32(gmax))
+        mean = deq.mean(axis=0)
+        step = (2.0 if grid == GRID_E2M1 else 1.0) * s
+        assert np.all(np.abs(mean - xv) <= step * (2.0 ** -9) + 4 * 0.5 * step / np.sqrt(n_blocks) + 1e-6)
+        # different blocks see different random bytes
+        assert len({bytes(q.codes[i]) for i in range(200)}) > 50
+        # and a different seed gives different draws, the same seed the same draws
+        q2 = oracle.quantize(bits, AXIS_ROW, rht_block=0, grid=grid, rounding=ROUND_SR, seed_sr=3)
+        q3 = oracle.quantize(bits, AXIS_ROW, rht_block=0, grid=grid, rounding=ROUND_SR, seed_sr=2)
+        assert not np.array_equal(q.codes, q2.codes) and np.array_equal(q.codes, q3.codes)
+
+
+# ------------------------------------------------------------------ the blockwise quantizer (Sec. 2.1, Sec. 4)
+
+def _rand_bits(rows, cols, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    return bf16_bits(rng.standard_normal((rows, cols)) * scale)
+
+
+@pytest.mark.parametrize("grid,gmax", [(GRID_INT4, 7.0), (GRID_E1M2, 1.75), (GRID_E2M1, 6.0)])
+def test_scale_is_amax_over_gmax_and_top_code_is_used(grid, gmax):
+    bits = _rand_bits(48, 64, 21, 0.37)
+    q = oracle.quantize(bits, AXIS_ROW, rht_block=0, grid=grid)
+    amax = np.abs(bf16_vals(bits)).reshape(48, 4, 16).max(axis=2)
+    assert np.array_equal(q.scales, (amax.astype(np.float32) / np.float32(gmax)).astype(np.float32))
+    lo, hi = q.codes & 0xF, q.codes >> 4
+    vals = np.vectorize(lambda n: abs(oracle.nibble_value(grid, int(n))))(np.stack([lo, hi], -1).reshape(48, 4, 16))
+    assert np.all(vals.max(axis=2) == gmax)          # no clipping and s = amax / g_max: the top level is always hit
+
+
+def test_e1m2_is_int4_with_scale_times_four():
+    bits = _rand_bits(32, 64, 22, 3.0)
+    for axis in (AXIS_ROW, AXIS_COL):
+        for rounding in (ROUND_RTNE, ROUND_SR):
+            a = oracle.quantize(bits, axis, 16, GRID_INT4, rounding, seed_rht=1, seed_sr=2)
+            b = oracle.quantize(bits, axis, 16, GRID_E1M2, rounding, seed_rht=1, seed_sr=2)
+            assert np.array_equal(b.scales, a.scales * np.float32(4.0))
+            assert np.array_equal(oracle.dequantize(a), oracle.dequantize(b))
+
+
+def test_rtne_error_bound_and_sr_error_bound():
+    """|x' - Q(x')| <= s/2 for RTNE on the uniform grid, < s for SR (x' the rotated value)."""
+    bits = _rand_bits(64, 64, 23)
+    mask = oracle.rht_sign_mask(1)
+    x = bf16_vals(bits).astype(np.float32)
+    xr = np.stack([oracle.rht16_f32(x[r, 16 * b:16 * b + 16], mask) for r in range(64) for b in range(4)])
+    xr = xr.reshape(64, 64).astype(np.float64)
+    for rounding, bound in ((ROUND_RTNE, 0.5), (ROUND_SR, 1.0)):
+        q = oracle.quantize(bits, AXIS_ROW, 16, GRID_INT4, rounding, seed_rht=1, seed_sr=9)
+        s = np.repeat(q.scales.astype(np.float64), 16, axis=1)
+        err = np.abs(oracle.dequantize(q) - xr)
+        assert np.all(err <= bound * s * (1 + 1e-6))
+
+
+def test_layout_of_row_and_col_variants():
+    """A single non-zero element: where its code and scale land, for both variants (RHT off)."""
+    rows, cols = 32, 48
+    for (r, c) in ((0, 0), (5, 17), (31, 47), (16, 32), (15, 31)):
+        x = np.zeros((rows, cols), dtype=np.float32)
+        x[r, c] = -3.0
+        bits = bf16_bits(x)
+        q = oracle.quantize(bits, AXIS_ROW, 0, GRID_INT4)
+        assert q.codes.shape == (rows, cols // 2) and q.scales.shape == (rows, cols // 16)
+        expect = np.zeros_like(q.codes)
+        expect[r, c // 2] = (0x9 if c % 2 == 0 else 0x90)     # -7 in two's complement = 0x9
+        assert np.array_equal(q.codes, expect)
+        es = np.zeros_like(q.scales)
+        es[r, c // 16] = np.float32(3.0) / np.float32(7.0)
+        assert np.array_equal(q.scales, es)
+        qc = oracle.quantize(bits, AXIS_COL, 0, GRID_INT4)
+        assert qc.codes.shape == (cols, rows // 2) and qc.scales.shape == (cols, rows // 16)
+        expect = np.zeros_like(qc.codes)
+        expect[c, r // 2] = (0x9 if r % 2 == 0 else 0x90)
+        assert np.array_equal(qc.codes, expect)
+        es = np.zeros_like(qc.scales)
+        es[c, r // 16] = np.float32(3.0) / np.float32(7.0)
+        assert np.array_equal(qc.scales, es)
+
+
+def test_col_variant_is_row_variant_of_the_transpose_with_its_own_sr_stream():
+    bits = _rand_bits(64, 48, 24)
+    bt = np.ascontiguousarray(bits.T)
+    for grid in (GRID_INT4, GRID_E2M1):
+        a = oracle.quantize(bits, AXIS_COL, 16, grid, ROUND_RTNE, seed_rht=1)
+        b = oracle.quantize(bt, AXIS_ROW, 16, grid, ROUND_RTNE, seed_rht=1)
+        assert np.array_equal(a.codes, b.codes) and np.array_equal(a.scales, b.scales)
+    a = oracle.quantize(bits, AXIS_COL, 16, GRID_INT4, ROUND_SR, seed_rht=1, seed_sr=2)
+    b = oracle.quantize(bt, AXIS_ROW, 16, GRID_INT4, ROUND_SR, seed_rht=1, seed_sr=2)
+    assert np.array_equal(a.scales, b.scales) and not np.array_equal(a.codes, b.codes)   # variant word differs
+
+
+def test_rotation_happens_before_scaling_and_rounding():
+    """Brute force on one block: rotate in FP64 with the matrix, then s = amax/7 and nearest integer."""
+    rng = np.random.default_rng(31)
+    mask = oracle.rht_sign_mask(7)
+    eps = np.array([-1.0 if (mask >> i) & 1 else 1.0 for i in range(16)])
+    Hp = np.diag(eps) @ oracle.hadamard_matrix(16)
+    x = rng.integers(-40, 40, size=(8, 16)).astype(np.float32)      # integers: FP32 butterflies are exact
+    q = oracle.quantize(bf16_bits(x), AXIS_ROW, 16, GRID_INT4, seed_rht=7, want_y=True)
+    xr = x.astype(np.float64) @ Hp
+    amax = np.abs(xr).max(axis=1)
+    assert np.array_equal(q.scales[:, 0], (amax.astype(np.float32) / np.float32(7)))
+    inv = np.float32(7) / amax.astype(np.float32)
+    y = (xr.astype(np.float32) * inv[:, None]).astype(np.float32)
+    assert np.array_equal(q.y, y)
+    codes = np.stack([q.codes & 0xF, q.codes >> 4], -1).reshape(8, 16).astype(np.int64)
+    codes = np.where(codes >= 8, codes - 16, codes)
+    assert np.array_equal(codes, np.rint(y.astype(np.float64)).astype(np.int64))
+
+
+def test_zero_and_tiny_blocks():
+    x = np.zeros((16, 32), dtype=np.float32)
+    x[3, 20] = 1e-35                                   # below 2^-100: treated as a zero block
+    x[4, 2] = 2.0
+    for fmt in (SCALE_FP32, SCALE_POW2):
+        q = oracle.quantize(bf16_bits(x), AXIS_ROW, 16, GRID_INT4, scale_fmt=fmt, seed_rht=1)
+        assert np.all(q.codes[3] == 0) and np.all(q.scales[3] == 0)
+        assert np.any(q.codes[4, :8] != 0) and q.scales[4, 0] > 0 and q.scales[4, 1] == 0
+        assert np.all(np.isfinite(oracle.dequantize(q)))
+
+
+def test_pow2_scale_is_the_next_power_of_two_and_is_idempotent():
+    bits = _rand_bits(32, 64, 25, 0.02)
+    q = oracle.quantize(bits, AXIS_ROW, 0, GRID_INT4, scale_fmt=SCALE_POW2)
+    f = oracle.quantize(bits, AXIS_ROW, 0, GRID_INT4, scale_fmt=SCALE_FP32)
+    m, e = np.frexp(q.scales)
+    assert np.all(m == 0.5)                                           # exact powers of two
+    assert np.all(q.scales >= f.scales) and np.all(q.scales < 2 * f.scales)
+    # q * 2^e is exactly BF16-representable, so quantizing the dequantized tensor reproduces codes and scales
+    deq = oracle.dequantize(q)
+    again = oracle.quantize(bf16_bits(deq), AXIS_ROW, 0, GRID_INT4, scale_fmt=SCALE_POW2)
+    assert np.array_equal(bf16_vals(bf16_bits(deq)), deq)
+    assert np.array_equal(again.codes, q.codes) and np.array_equal(again.scales, q.scales)
+
+
+def test_e4m3_helpers_round_trip():
+    vals = [oracle.e4m3_value(c) for c in range(0x7F)]
+    assert vals[0] == 0 and vals[1] == 2.0 ** -9 and vals[0x7E] == 448.0 and vals[0x38] == 1.0
+    assert all(b > a for a, b in zip(vals, vals[1:]))
+    for c in range(0x7F):
+        assert oracle.e4m3_encode(vals[c]) == c
+    assert oracle.e4m3_encode(1e9) == 0x7E and oracle.e4m3_encode(0.0) == 0
+    for c in range(1, 0x7E):                          # midpoints go to the even code
+        mid = (vals[c] + vals[c + 1]) / 2
+        assert oracle.e4m3_encode(mid) == (c if c % 2 == 0 else c + 1)
+
+
+def test_e4m3_tensor_scale_mode_brute_force():
+    bits = _rand_bits(16, 64, 26)
+    x = bf16_vals(bits)
+    ts = float(np.float32(4 * np.abs(x).max() / (7 * 448)))
+    q = oracle.quantize(bits, AXIS_ROW, 16, GRID_INT4, scale_fmt=SCALE_E4M3_TENSOR, seed_rht=1, tensor_scale=ts)
+    assert q.scales.dtype == np.uint8
+    mask = oracle.rht_sign_mask(1)
+    deq = oracle.dequantize(q)
+    for r in range(16):
+        for b in range(4):
+            xr = oracle.rht16_f32(x[r, 16 * b:16 * b + 16].astype(np.float32), mask)
+            z = np.float32(np.abs(xr).max()) / np.float32(7)
+            byte = oracle.e4m3_encode(float(z / np.float32(ts)))
+            assert q.scales[r, b] == byte
+            s = np.float32(ts) * np.float32(oracle.e4m3_value(byte))
+            y = xr * (np.float32(1) / s)
+            expect = np.clip(np.rint(y.astype(np.float64)), -7, 7) * float(s)
+            assert np.array_equal(deq[r, 16 * b:16 * b + 16], expect)
+
+
+# ------------------------------------------------------------------ GEMM on dequantized operands (Sec. 2.2)
+
+def test_gemm_reduces_to_integer_matmul_when_scales_are_one():
+    rng = np.random.default_rng(41)
+    M, N, K = 24, 40, 64
+    qa = rng.integers(-7, 8, size=(M, K))
+    qb = rng.integers(-7, 8, size=(N, K))
+    qa[:, ::16] = 7                                   # amax = 7 in every block -> scale exactly 1 (RHT off)
+    qb[:, ::16] = -7
+    A = oracle.quantize(bf16_bits(qa), AXIS_ROW, 0, GRID_INT4)
+    B = oracle.quantize(bf16_bits(qb), AXIS_ROW, 0, GRID_INT4)
+    assert np.all(A.scales == 1) and np.all(B.scales == 1)
+    Cm, S = oracle.gemm(A, B)
+    assert np.array_equal(Cm, (qa @ qb.T).astype(np.float64))
+    assert np.array_equal(S, (np.abs(qa) @ np.abs(qb).T).astype(np.float64))
+    # not symmetric in its operands: C is [M][N] with A's rows first
+    assert Cm.shape == (M, N)
+    c, s = oracle.gemm_sampled(A, B, [0, 3, 23], [0, 39, 7])
+    assert np.array_equal(c, Cm[[0, 3, 23], [0, 39, 7]]) and np.array_equal(s, S[[0, 3, 23], [0, 39, 7]])
+    c2, _ = oracle.gemm_sampled(A, B, [3], [39], 16, 48)
+    assert c2[0] == float(qa[3, 16:48] @ qb[39, 16:48])
+
+
+def test_gemm_one_hot_operands_pick_out_entries():
+    K = 32
+    a = np.zeros((16, K), dtype=np.float32)
+    b = np.zeros((16, K), dtype=np.float32)
+    for i in range(16):
+        a[i, i] = 2.0
+        b[i, (i + 1) % 16] = 3.0
+    A = oracle.quantize(bf16_bits(a), AXIS_ROW, 0, GRID_INT4, scale_fmt=SCALE_POW2)
+    B = oracle.quantize(bf16_bits(b), AXIS_ROW, 0, GRID_INT4, scale_fmt=SCALE_POW2)
+    Cm, _ = oracle.gemm(A, B)
+    # POW2 scale of amax 2 is 2/7 -> 0.5, code 4; of amax 3: 3/7 -> 0.5, code 6: values are exact
+    expect = np.zeros((16, 16))
+    for i in range(16):
+        expect[(i + 1) % 16, i] = 6.0
+    assert np.array_equal(Cm, expect)
+
+
+def test_freivalds_and_closeness_to_the_unquantized_product():
+    rng = np.random.default_rng(43)
+    M, N, K = 48, 32, 128
+    X = rng.standard_normal((M, K))
+    W = rng.standard_normal((N, K)) * 0.02
+    xb, wb = bf16_bits(X), bf16_bits(W)
+    exact = bf16_vals(xb) @ bf16_vals(wb).T
+    errs = {}
+    for grid in (GRID_INT4, GRID_E2M1):
+        A = oracle.quantize(xb, AXIS_ROW, 16, grid, seed_rht=1)
+        B = oracle.quantize(wb, AXIS_ROW, 16, grid, seed_rht=1)
+        Cm, S = oracle.gemm(A, B)
+        v = rng.standard_normal(N)
+        lhs = Cm @ v
+        rhs = oracle.dequantize(A) @ (oracle.dequantize(B).T @ v)
+        assert np.max(np.abs(lhs - rhs)) <= 1e-12 * np.max(S)
+        errs[grid] = np.linalg.norm(Cm - exact) / np.linalg.norm(exact)
+        assert errs[grid] < 0.25        # same rotation on both operands: only quantization error remains
+    # a different rotation on the two operands breaks the identity (XH')(WH')^T = XW^T
+    A = oracle.quantize(xb, AXIS_ROW, 16, GRID_INT4, seed_rht=1)
+    B = oracle.quantize(wb, AXIS_ROW, 16, GRID_INT4, seed_rht=5)
+    assert oracle.rht_sign_mask(1) != oracle.rht_sign_mask(5)
+    Cm, _ = oracle.gemm(A, B)
+    assert np.linalg.norm(Cm - exact) / np.linalg.norm(exact) > 0.5
