@@ -1,0 +1,178 @@
+/*
+ * ufp4.h — C ABI of libufp4: the UFP4 training hot path on NVIDIA B200 (sm_100a).
+ *
+ * Two operations, as the paper states them:
+ *   1. the blockwise quantizer of Sec. 2.1 (s_B = max|x_j| / g_max, q_i = rho_G(x_i / s_B), rho_G = RTNE or SR) fused
+ *      with the 16-point Random Hadamard Transform of Sec. 2.2 (H'_16 = S_16 H_16), in the configuration of
+ *      Sec. 4 / Table 1: 1x16 blocks, one scale per block, RHT block 16, RTNE for X and W, SR for dY;
+ *   2. the low-precision GEMM of Sec. 2.2, Y^ = Q_G(X H') Q_G(W H')^T, for the three training products fwd_y, bwd_dx
+ *      and bwd_dw, each reducing over the dimension its operands were rotated and blocked along.
+ *
+ * Conventions
+ *   - Every data pointer is DEVICE memory owned and sized by the caller unless a parameter says "host".  The library
+ *     allocates no device memory and keeps no per-call state.  Work is enqueued on the caller's CUDA stream
+ *     (a cudaStream_t passed as void*; NULL = the default stream) and the call returns without synchronizing.
+ *   - Errors the host can see (null pointers, shapes, alignment, enums, too-small workspace) return a negative
+ *     ufp4_status and launch nothing.  Conditions only the device can see set bits in *dev_status (device int32,
+ *     optional): UFP4_DEV_NONFINITE, UFP4_DEV_EXP_WINDOW, UFP4_DEV_WAIT_TIMEOUT.  Bits are OR-ed in, never cleared.
+ *   - A quantized tensor is logically [rows][k] with k the reduction dimension; codes are packed two per byte along k
+ *     (element 2j in bits 3:0 of byte j, element 2j+1 in bits 7:4); there is one scale per 16 consecutive k.
+ *   - All three training GEMMs are the same contraction C[m][n] = sum_k A[m][k] * B[n][k] on k-contiguous operands:
+ *       fwd_y : A = rows variant of X  [T][K],  B = row variant of W  [N][K]   -> Y  [T][N]
+ *       bwd_dx: A = row variant of dY  [T][N],  B = col variant of W  [K][N]   -> dX [T][K]
+ *       bwd_dw: A = col variant of dY  [N][T],  B = col variant of X  [K][T]   -> dW [N][K]
+ *     Both operands of a product must have been quantized with the same seed_rht and rht_block along the shared
+ *     dimension (Sec. 2.2: the identity X W^T = (X H')(W H')^T needs the same H'); the library cannot check this.
+ */
+#ifndef UFP4_H_
+#define UFP4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    UFP4_OK = 0,
+    UFP4_ERR_NULL = -1,        /* a required pointer is NULL */
+    UFP4_ERR_SHAPE = -2,       /* a dimension is non-positive or not a multiple of what the operation needs */
+    UFP4_ERR_ALIGN = -3,       /* a pointer or leading dimension breaks the stated alignment */
+    UFP4_ERR_ENUM = -4,        /* an enum value is out of range */
+    UFP4_ERR_UNSUPPORTED = -5, /* a valid combination this build does not implement */
+    UFP4_ERR_CUDA = -6,        /* a CUDA runtime call failed (launch error, no sm_100 device, ...) */
+    UFP4_ERR_WORKSPACE = -7    /* workspace missing or smaller than ufp4_gemm_workspace_bytes() */
+} ufp4_status;
+
+/* Data-element grids (Sec. 2.1; Sec. 3.1 prints the E2M1 magnitudes).  INT4 and E1M2 are the same uniform grid:
+ * INT4 stores q in [-7,7] as a two's-complement nibble with g_max = 7; E1M2 stores sign|e|mm with values q/4 and
+ * g_max = 1.75, so its block scale is exactly 4x the INT4 one.  E2M1 is the comparison grid {0,.5,1,1.5,2,3,4,6}
+ * stored as sign|ee|m.  Zero is always encoded as nibble 0x0. */
+typedef enum { UFP4_GRID_INT4 = 0, UFP4_GRID_E1M2 = 1, UFP4_GRID_E2M1 = 2 } ufp4_grid;
+
+/* Rounding rule rho_G (Sec. 2.1).  RTNE: nearest level, ties to the even code.  SR: between neighbouring levels
+ * g_a <= t < g_b the upper one is taken with probability (t - g_a)/(g_b - g_a), resolved to 1/256 by one random byte
+ * per element from Philox4x32-10 keyed by seed_sr and the block index (Table 1: SR on dY only). */
+typedef enum { UFP4_ROUND_RTNE = 0, UFP4_ROUND_SR = 1 } ufp4_round;
+
+/* Which dimension the 16-element blocks (and the RHT) run along (Sec. 2.2, last paragraph: the reduction dimension
+ * of the product the tensor feeds).  ROW: along the last dimension.  COL: along the first dimension, output stored
+ * transposed.  BOTH: both variants from one pass over the input. */
+typedef enum { UFP4_AXIS_ROW = 0, UFP4_AXIS_COL = 1, UFP4_AXIS_BOTH = 2 } ufp4_axis;
+
+/* Block-scale format.  FP32: s = RN(amax / g_max), Table 1's "FP32 single-level".  POW2: that value rounded up to a
+ * power of two, still stored as FP32 (Sec. 4 leaves the scale hierarchy open "depending on hardware efficiency"); it
+ * is the format the tensor-core GEMM path folds into its 8-bit operands exactly.  E4M3_TENSOR: an E4M3 byte per
+ * block times one FP32 per tensor (the two-level layout Sec. 2.1's footnote attributes to NVFP4). */
+typedef enum { UFP4_SCALE_FP32 = 0, UFP4_SCALE_POW2 = 1, UFP4_SCALE_E4M3_TENSOR = 2 } ufp4_scale_fmt;
+
+/* Which training product a GEMM call computes.  All are C = A B^T on k-contiguous operands; the value matters only to
+ * the grouped call, where fwd_y / bwd_dx split the rows of A (and C) by group and bwd_dw splits the reduction. */
+typedef enum { UFP4_FWD_Y = 0, UFP4_BWD_DX = 1, UFP4_BWD_DW = 2 } ufp4_layout;
+
+/* Bits of *dev_status. */
+enum {
+    UFP4_DEV_NONFINITE = 1,    /* a block held Inf/NaN: its codes and scale are unspecified */
+    UFP4_DEV_EXP_WINDOW = 2,   /* tensor-core GEMM: a block scale lay outside the exponent window of its row and was
+                                  flushed to zero; re-run with the exact path (see ufp4_gemm) */
+    UFP4_DEV_WAIT_TIMEOUT = 4  /* a bounded pipeline wait inside a kernel gave up; the output is invalid */
+};
+
+/* A quantized tensor (device pointers, caller-owned). */
+typedef struct ufp4_qtensor {
+    void *codes;               /* uint8 [rows][ld_codes_bytes]; the first k/2 bytes of a row are used; 16-B aligned */
+    void *scales;              /* float [rows][ld_scales] (FP32, POW2) or uint8 [rows][ld_scales] (E4M3_TENSOR)      */
+    const float *tensor_scale; /* device pointer to one float; E4M3_TENSOR only (input to the quantizer), else NULL  */
+    int64_t rows;              /* logical rows                                                                       */
+    int64_t k;                 /* reduction dimension, multiple of 16                                                */
+    int64_t ld_codes_bytes;    /* row pitch of codes in bytes, multiple of 16, >= k/2                                */
+    int64_t ld_scales;         /* row pitch of scales in elements, >= k/16                                           */
+    int32_t grid;              /* ufp4_grid                                                                          */
+    int32_t scale_fmt;         /* ufp4_scale_fmt                                                                     */
+} ufp4_qtensor;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int ufp4_version(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char *ufp4_status_string(int status);
+
+/* The 16 RHT signs of a seed (host computation): bit i set means eps_i = -1 (Sec. 2.2, S_16 = diag(eps)).
+ * Bits are the low 16 bits of word 0 of Philox4x32-10 with counter (0,0,0,0x52485400) and key (lo32, hi32) of seed. */
+uint32_t ufp4_rht_sign_mask(uint64_t seed_rht);
+
+/* Densely packed sizes of a [rows][k] quantized tensor (ld_codes_bytes = k/2 rounded up to 16, ld_scales = k/16). */
+int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t *codes_bytes, size_t *scales_bytes);
+
+/*
+ * Fused RHT + blockwise quantizer (Sec. 2.1 quantizer; Sec. 2.2 RHT; Sec. 4 / Table 1 settings; Sec. 5.5 describes
+ * the fusion: rotate before scale estimation and packing, no rotated tensor is materialised).
+ *
+ *   x          BF16 [rows][cols], row pitch ld elements; 16-B aligned, ld % 8 == 0
+ *   axis       ROW needs cols % 16 == 0 and fills *out_row = [rows][cols];
+ *              COL needs rows % 16 == 0 and cols % 16 == 0 and fills *out_col = [cols][rows];
+ *              BOTH fills both from a single read of x
+ *   rht_block  0 (no rotation) or 16
+ *   seed_rht   selects the sign vector (ufp4_rht_sign_mask); along COL the sign of row r is eps_(r mod 16)
+ *   seed_sr    key of the SR random bytes; counter = (lo32(b), hi32(b), variant, 0x53520000), b = index of the block in
+ *              the variant's dense [rows][k/16] scale array, variant 0 = row, 1 = col
+ *   out_row / out_col   describe caller-allocated outputs; rows, k, grid and scale_fmt must match the call, and for
+ *              E4M3_TENSOR tensor_scale must point at the FP32 tensor scale to use
+ *
+ * Per block, in FP32: v = x (o) eps; butterfly stages h = 1,2,4,8; x' = v/4; amax = max|x'|; s = RN(amax/g_max);
+ * y = RN(x' * RN(g_max/amax)); q = rho_G(y).  Blocks with amax == 0 or amax < 2^-100 store scale 0 and codes 0.
+ * Inputs must be finite (else UFP4_DEV_NONFINITE) and |x'| <= 2^120.  Output is bit-reproducible.
+ */
+int ufp4_quantize(const void *x, int64_t rows, int64_t cols, int64_t ld, int axis, int rht_block, int grid,
+                  int rounding, int scale_fmt, uint64_t seed_rht, uint64_t seed_sr, const ufp4_qtensor *out_row,
+                  const ufp4_qtensor *out_col, int32_t *dev_status, void *stream);
+
+/*
+ * The same quantizer over a batch of equally shaped matrices x[e] = x + e * batch_stride (elements), e.g. the expert
+ * weights [E][N][K] of an MoE layer (Sec. 5 trains MoE models; the quantizer itself is Sec. 2.1 / 2.2 as above).
+ * Outputs are stacked along rows: *out_row = [batch * rows][cols], *out_col = [batch * cols][rows] (matrix e owns rows
+ * [e * cols, (e+1) * cols) of it).  batch_stride % 8 == 0.  RTNE only (weights are never stochastically rounded,
+ * Table 1); SR returns UFP4_ERR_UNSUPPORTED when batch > 1.
+ */
+int ufp4_quantize_batched(const void *x, int64_t batch, int64_t batch_stride, int64_t rows, int64_t cols, int64_t ld,
+                          int axis, int rht_block, int grid, int rounding, int scale_fmt, uint64_t seed_rht,
+                          uint64_t seed_sr, const ufp4_qtensor *out_row, const ufp4_qtensor *out_col,
+                          int32_t *dev_status, void *stream);
+
+/* Workspace the GEMM calls need for these operands (0 for the exact path). */
+size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path);
+
+/* GEMM paths.  AUTO picks TENSOR when both operands use POW2 scales and the shape fits its tiles, else EXACT.
+ * EXACT: integer block partials promoted with the two FP32 block scales; valid for every grid and scale format.
+ * TENSOR: tcgen05 / TMEM kernel on 8-bit floating-point operands into which code x 2^e is folded exactly (POW2
+ * scales only); blocks whose exponent lies outside a row's window set UFP4_DEV_EXP_WINDOW. */
+typedef enum { UFP4_PATH_AUTO = 0, UFP4_PATH_EXACT = 1, UFP4_PATH_TENSOR = 2 } ufp4_gemm_path;
+
+/*
+ * C[m][n] = sum_k a[m][k] * b[n][k], a = value(code) * scale (Sec. 2.2, Y^ = Q_G(XH') Q_G(WH')^T).
+ *   A [M][K], B [N][K] quantized tensors with equal k; grids may differ
+ *   C       FP32 (c_is_bf16 == 0) or BF16 [M][ldc], ldc in elements, 16-B aligned rows
+ *   workspace / workspace_bytes   >= ufp4_gemm_workspace_bytes(A, B, path); may be NULL/0 when that is 0
+ * Accumulation is FP32 or better; the result differs from the exact sum by at most 1e-5 * sum_k |a_k b_k|.
+ */
+int ufp4_gemm(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int layout, int path,
+              void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/*
+ * MoE-grouped variant: one call for all experts.  offsets is a DEVICE int64 [num_groups+1] array of row offsets
+ * (offsets[0] = 0, every offset a multiple of 128; padding rows must hold zero codes or zero scales), and
+ * host_offsets the same values in HOST memory (the launch geometry is sized from them).
+ *   FWD_Y, BWD_DX: A [total][K] with rows grouped; B [num_groups * N][K] (expert e owns rows [e*N, (e+1)*N));
+ *                  C [total][N]: C[t][:] = A[t][:] . B_e(t)^T
+ *   BWD_DW:        A [N][total], B [Kout][total] (reduction dimension grouped); C [num_groups * N][Kout]:
+ *                  C_e = sum over k in [offsets[e], offsets[e+1]) of A[:,k] B[:,k]^T; an empty group writes zeros
+ */
+int ufp4_gemm_grouped(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int layout,
+                      int path, const int64_t *offsets, const int64_t *host_offsets, int num_groups, int64_t group_n,
+                      void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UFP4_H_ */

@@ -1,0 +1,224 @@
+"""ctypes binding of libufp4.so (declared in include/ufp4.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.  PyTorch supplies device
+memory and streams.  There is no CPU fallback; if the library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+GRID_INT4, GRID_E1M2, GRID_E2M1 = 0, 1, 2
+ROUND_RTNE, ROUND_SR = 0, 1
+AXIS_ROW, AXIS_COL, AXIS_BOTH = 0, 1, 2
+SCALE_FP32, SCALE_POW2, SCALE_E4M3_TENSOR = 0, 1, 2
+FWD_Y, BWD_DX, BWD_DW = 0, 1, 2
+PATH_AUTO, PATH_EXACT, PATH_TENSOR = 0, 1, 2
+DEV_NONFINITE, DEV_EXP_WINDOW, DEV_WAIT_TIMEOUT = 1, 2, 4
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libufp4.so")
+
+EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_qtensor_bytes", "ufp4_quantize",
+           "ufp4_quantize_batched", "ufp4_gemm_workspace_bytes", "ufp4_gemm", "ufp4_gemm_grouped"]
+
+
+class _QTensorStruct(C.Structure):
+    _fields_ = [("codes", C.c_void_p), ("scales", C.c_void_p), ("tensor_scale", C.c_void_p),
+                ("rows", C.c_int64), ("k", C.c_int64), ("ld_codes_bytes", C.c_int64), ("ld_scales", C.c_int64),
+                ("grid", C.c_int32), ("scale_fmt", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libufp4.so (once).  Raises if it has not been built: there is no other implementation to fall back to."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2606_20381_b200.build` "
+                               "(the UFP4 path has no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i64, u64, i32, sz = C.c_void_p, C.c_int64, C.c_uint64, C.c_int, C.c_size_t
+        qp = C.POINTER(_QTensorStruct)
+        L.ufp4_version.restype = i32
+        L.ufp4_version.argtypes = []
+        L.ufp4_status_string.restype = C.c_char_p
+        L.ufp4_status_string.argtypes = [i32]
+        L.ufp4_rht_sign_mask.restype = C.c_uint32
+        L.ufp4_rht_sign_mask.argtypes = [u64]
+        L.ufp4_qtensor_bytes.restype = i32
+        L.ufp4_qtensor_bytes.argtypes = [i64, i64, i32, C.POINTER(sz), C.POINTER(sz)]
+        L.ufp4_quantize.restype = i32
+        L.ufp4_quantize.argtypes = [vp, i64, i64, i64, i32, i32, i32, i32, i32, u64, u64, qp, qp, vp, vp]
+        L.ufp4_quantize_batched.restype = i32
+        L.ufp4_quantize_batched.argtypes = [vp, i64, i64, i64, i64, i64, i32, i32, i32, i32, i32, u64, u64, qp, qp, vp, vp]
+        L.ufp4_gemm_workspace_bytes.restype = sz
+        L.ufp4_gemm_workspace_bytes.argtypes = [qp, qp, i32]
+        L.ufp4_gemm.restype = i32
+        L.ufp4_gemm.argtypes = [qp, qp, vp, i64, i32, i32, i32, vp, sz, vp, vp]
+        L.ufp4_gemm_grouped.restype = i32
+        L.ufp4_gemm_grouped.argtypes = [qp, qp, vp, i64, i32, i32, i32, vp, vp, i32, i64, vp, sz, vp, vp]
+        _lib = L
+    return _lib
+
+
+class Ufp4Error(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(f"libufp4 status {status}: {lib().ufp4_status_string(status).decode()}")
+
+
+def _check(status: int):
+    if status != 0:
+        raise Ufp4Error(status)
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+@dataclass
+class QTensor:
+    """A quantized tensor on the device: logical [rows][k], k the reduction dimension."""
+    codes: torch.Tensor                     # uint8 [rows][ld_codes_bytes]
+    scales: torch.Tensor                    # float32 or uint8 [rows][k/16]
+    grid: int
+    scale_fmt: int
+    k: int
+    tensor_scale: torch.Tensor | None = None   # float32 [1] on the device (E4M3_TENSOR only)
+
+    @property
+    def rows(self) -> int:
+        return self.codes.shape[0]
+
+    def struct(self) -> _QTensorStruct:
+        return _QTensorStruct(self.codes.data_ptr(), self.scales.data_ptr(),
+                              self.tensor_scale.data_ptr() if self.tensor_scale is not None else None,
+                              self.rows, self.k, self.codes.stride(0), self.scales.stride(0), self.grid, self.scale_fmt)
+
+    def packed_codes(self) -> torch.Tensor:
+        """uint8 [rows][k/2] view without row padding."""
+        return self.codes[:, : self.k // 2]
+
+    def row_slice(self, r0: int, r1: int) -> "QTensor":
+        return QTensor(self.codes[r0:r1], self.scales[r0:r1], self.grid, self.scale_fmt, self.k, self.tensor_scale)
+
+
+def rht_sign_mask(seed: int) -> int:
+    return int(lib().ufp4_rht_sign_mask(seed))
+
+
+def alloc_qtensor(rows: int, k: int, grid: int, scale_fmt: int, device, tensor_scale=None) -> QTensor:
+    cb, sb = C.c_size_t(), C.c_size_t()
+    _check(lib().ufp4_qtensor_bytes(rows, k, scale_fmt, C.byref(cb), C.byref(sb)))
+    ld = cb.value // rows
+    codes = torch.empty(rows, ld, dtype=torch.uint8, device=device)
+    sdt = torch.uint8 if scale_fmt == SCALE_E4M3_TENSOR else torch.float32
+    scales = torch.empty(rows, k // 16, dtype=sdt, device=device)
+    ts = None
+    if scale_fmt == SCALE_E4M3_TENSOR:
+        if tensor_scale is None:
+            raise ValueError("E4M3_TENSOR needs a tensor_scale")
+        ts = tensor_scale if isinstance(tensor_scale, torch.Tensor) else torch.tensor(
+            [tensor_scale], dtype=torch.float32, device=device)
+    return QTensor(codes, scales, grid, scale_fmt, k, ts)
+
+
+def quantize(x: torch.Tensor, axis: int = AXIS_BOTH, rht_block: int = 16, grid: int = GRID_INT4,
+             rounding: int = ROUND_RTNE, scale_fmt: int = SCALE_FP32, seed_rht: int = 0, seed_sr: int = 0,
+             tensor_scale=None, out_row: QTensor | None = None, out_col: QTensor | None = None,
+             dev_status: torch.Tensor | None = None, stream=None):
+    """ufp4_quantize on a BF16 CUDA matrix [rows][cols]; returns (row variant or None, col variant or None)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    if axis != AXIS_COL and out_row is None:
+        out_row = alloc_qtensor(rows, cols, grid, scale_fmt, x.device, tensor_scale)
+    if axis != AXIS_ROW and out_col is None:
+        out_col = alloc_qtensor(cols, rows, grid, scale_fmt, x.device, tensor_scale)
+    sr = out_row.struct() if axis != AXIS_COL else None
+    sc = out_col.struct() if axis != AXIS_ROW else None
+    _check(lib().ufp4_quantize(x.data_ptr(), rows, cols, x.stride(0), axis, rht_block, grid, rounding, scale_fmt,
+                               seed_rht, seed_sr, C.byref(sr) if sr is not None else None,
+                               C.byref(sc) if sc is not None else None,
+                               dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
+    return (out_row if axis != AXIS_COL else None), (out_col if axis != AXIS_ROW else None)
+
+
+def quantize_batched(x: torch.Tensor, axis: int = AXIS_BOTH, rht_block: int = 16, grid: int = GRID_INT4,
+                     rounding: int = ROUND_RTNE, scale_fmt: int = SCALE_FP32, seed_rht: int = 0, seed_sr: int = 0,
+                     tensor_scale=None, out_row: QTensor | None = None, out_col: QTensor | None = None,
+                     dev_status: torch.Tensor | None = None, stream=None):
+    """ufp4_quantize_batched on a BF16 CUDA tensor [batch][rows][cols]; outputs stacked along rows."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 3 and x.stride(2) == 1
+    batch, rows, cols = x.shape
+    if axis != AXIS_COL and out_row is None:
+        out_row = alloc_qtensor(batch * rows, cols, grid, scale_fmt, x.device, tensor_scale)
+    if axis != AXIS_ROW and out_col is None:
+        out_col = alloc_qtensor(batch * cols, rows, grid, scale_fmt, x.device, tensor_scale)
+    sr = out_row.struct() if axis != AXIS_COL else None
+    sc = out_col.struct() if axis != AXIS_ROW else None
+    _check(lib().ufp4_quantize_batched(x.data_ptr(), batch, x.stride(0), rows, cols, x.stride(1), axis, rht_block, grid,
+                                       rounding, scale_fmt, seed_rht, seed_sr,
+                                       C.byref(sr) if sr is not None else None,
+                                       C.byref(sc) if sc is not None else None,
+                                       dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
+    return (out_row if axis != AXIS_COL else None), (out_col if axis != AXIS_ROW else None)
+
+
+def gemm_workspace_bytes(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:
+    sa, sb = A.struct(), B.struct()
+    return int(lib().ufp4_gemm_workspace_bytes(C.byref(sa), C.byref(sb), path))
+
+
+def _workspace(A, B, path, workspace):
+    need = gemm_workspace_bytes(A, B, path)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=A.codes.device)
+    return workspace
+
+
+def gemm(A: QTensor, B: QTensor, out: torch.Tensor | None = None, out_bf16: bool = False, layout: int = FWD_Y,
+         path: int = PATH_AUTO, workspace: torch.Tensor | None = None, dev_status: torch.Tensor | None = None,
+         stream=None) -> torch.Tensor:
+    """ufp4_gemm: C[m][n] = sum_k a[m][k] b[n][k] for quantized A [M][K], B [N][K]."""
+    if out is None:
+        out = torch.empty(A.rows, B.rows, dtype=torch.bfloat16 if out_bf16 else torch.float32, device=A.codes.device)
+    assert out.is_cuda and out.stride(1) == 1
+    workspace = _workspace(A, B, path, workspace)
+    sa, sb = A.struct(), B.struct()
+    _check(lib().ufp4_gemm(C.byref(sa), C.byref(sb), out.data_ptr(), out.stride(0), int(out.dtype == torch.bfloat16),
+                           layout, path, workspace.data_ptr() if workspace is not None else None,
+                           workspace.numel() if workspace is not None else 0,
+                           dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
+    return out
+
+
+def gemm_grouped(A: QTensor, B: QTensor, offsets_dev: torch.Tensor, offsets_host: torch.Tensor, group_n: int,
+                 layout: int, out: torch.Tensor | None = None, out_bf16: bool = False, path: int = PATH_AUTO,
+                 workspace: torch.Tensor | None = None, dev_status: torch.Tensor | None = None,
+                 stream=None) -> torch.Tensor:
+    """ufp4_gemm_grouped (see include/ufp4.h for the operand layouts of each product)."""
+    assert offsets_dev.is_cuda and offsets_dev.dtype == torch.int64 and offsets_dev.is_contiguous()
+    assert (not offsets_host.is_cuda) and offsets_host.dtype == torch.int64 and offsets_host.is_contiguous()
+    G = offsets_host.numel() - 1
+    if out is None:
+        dt = torch.bfloat16 if out_bf16 else torch.float32
+        if layout == BWD_DW:
+            out = torch.empty(G * A.rows, B.rows, dtype=dt, device=A.codes.device)
+        else:
+            out = torch.empty(A.rows, group_n, dtype=dt, device=A.codes.device)
+    workspace = _workspace(A, B, path, workspace)
+    sa, sb = A.struct(), B.struct()
+    _check(lib().ufp4_gemm_grouped(C.byref(sa), C.byref(sb), out.data_ptr(), out.stride(0),
+                                   int(out.dtype == torch.bfloat16), layout, path, offsets_dev.data_ptr(),
+                                   offsets_host.data_ptr(), G, group_n,
+                                   workspace.data_ptr() if workspace is not None else None,
+                                   workspace.numel() if workspace is not None else 0,
+                                   dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
+    return out

@@ -1,0 +1,119 @@
+// Host-side entry points of libufp4 that are not tied to one kernel file: version, status strings, size helpers and
+// the GEMM dispatch (argument validation, path selection).
+#include "common.cuh"
+
+namespace ufp4 {
+int gemm_exact_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
+                      int64_t M, int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n,
+                      void *stream);
+size_t gemm_tensor_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
+bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
+int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
+                       int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
+                       int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                       void *stream);
+
+static int check_operand(const ufp4_qtensor *q) {
+    if (!q || !q->codes || !q->scales) return UFP4_ERR_NULL;
+    if (q->grid < 0 || q->grid > 2 || q->scale_fmt < 0 || q->scale_fmt > 2) return UFP4_ERR_ENUM;
+    if (q->rows < 1 || q->k < 16 || q->k % 16 != 0) return UFP4_ERR_SHAPE;
+    if (q->ld_codes_bytes < q->k / 2 || q->ld_codes_bytes % 16 != 0 || q->ld_scales < q->k / 16) return UFP4_ERR_ALIGN;
+    if (!aligned_to(q->codes, 16)) return UFP4_ERR_ALIGN;
+    if (q->scale_fmt != UFP4_SCALE_E4M3_TENSOR && !aligned_to(q->scales, 4)) return UFP4_ERR_ALIGN;
+    if (q->scale_fmt == UFP4_SCALE_E4M3_TENSOR && !q->tensor_scale) return UFP4_ERR_NULL;
+    return UFP4_OK;
+}
+
+static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int path,
+                         int mode, int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
+                         int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                         void *stream) {
+    if (path < 0 || path > 2) return UFP4_ERR_ENUM;
+    if (!C) return UFP4_ERR_NULL;
+    if (ldc < N) return UFP4_ERR_SHAPE;
+    if (!aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
+    bool tensor_ok = gemm_tensor_supported(A, B, M, N, K, mode);
+    if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_EXACT || !tensor_ok)
+        return gemm_exact_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, stream);
+    size_t need = gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
+    if (!workspace || workspace_bytes < need) {
+        if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
+        return gemm_exact_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, stream);
+    }
+    return gemm_tensor_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
+                              workspace, workspace_bytes, dev_status, stream);
+}
+
+}  // namespace ufp4
+
+extern "C" int ufp4_version(void) { return 100; }
+
+extern "C" const char *ufp4_status_string(int status) {
+    switch (status) {
+        case UFP4_OK: return "ok";
+        case UFP4_ERR_NULL: return "a required pointer is NULL";
+        case UFP4_ERR_SHAPE: return "bad shape: a dimension is non-positive or not a multiple of what the operation needs";
+        case UFP4_ERR_ALIGN: return "bad alignment of a pointer or leading dimension";
+        case UFP4_ERR_ENUM: return "enum value out of range";
+        case UFP4_ERR_UNSUPPORTED: return "combination not supported by this build";
+        case UFP4_ERR_CUDA: return "a CUDA runtime call failed";
+        case UFP4_ERR_WORKSPACE: return "workspace missing or too small";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t *codes_bytes, size_t *scales_bytes) {
+    if (!codes_bytes || !scales_bytes) return UFP4_ERR_NULL;
+    if (rows < 1 || k < 16 || k % 16 != 0) return UFP4_ERR_SHAPE;
+    if (scale_fmt < 0 || scale_fmt > 2) return UFP4_ERR_ENUM;
+    int64_t ld = (k / 2 + 15) / 16 * 16;
+    *codes_bytes = (size_t)(rows * ld);
+    *scales_bytes = (size_t)(rows * (k / 16) * (scale_fmt == UFP4_SCALE_E4M3_TENSOR ? 1 : 4));
+    return UFP4_OK;
+}
+
+extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path) {
+    if (!A || !B || path == UFP4_PATH_EXACT) return 0;
+    if (A->scale_fmt != UFP4_SCALE_POW2 || B->scale_fmt != UFP4_SCALE_POW2) return 0;
+    return ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
+}
+
+extern "C" int ufp4_gemm(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int layout,
+                         int path, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
+    int rc = ufp4::check_operand(A);
+    if (rc != UFP4_OK) return rc;
+    rc = ufp4::check_operand(B);
+    if (rc != UFP4_OK) return rc;
+    if (layout < 0 || layout > 2) return UFP4_ERR_ENUM;
+    if (A->k != B->k) return UFP4_ERR_SHAPE;
+    return ufp4::gemm_dispatch(A, B, C, ldc, c_is_bf16, path, 0, A->rows, B->rows, A->k, nullptr, nullptr, 1, B->rows,
+                               workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" int ufp4_gemm_grouped(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16,
+                                 int layout, int path, const int64_t *offsets, const int64_t *host_offsets,
+                                 int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes,
+                                 int32_t *dev_status, void *stream) {
+    int rc = ufp4::check_operand(A);
+    if (rc != UFP4_OK) return rc;
+    rc = ufp4::check_operand(B);
+    if (rc != UFP4_OK) return rc;
+    if (layout < 0 || layout > 2) return UFP4_ERR_ENUM;
+    if (!offsets || !host_offsets) return UFP4_ERR_NULL;
+    if (num_groups < 1 || A->k != B->k) return UFP4_ERR_SHAPE;
+    if (host_offsets[0] != 0) return UFP4_ERR_SHAPE;
+    for (int g = 0; g < num_groups; ++g)
+        if (host_offsets[g + 1] < host_offsets[g] || host_offsets[g + 1] % 128 != 0) return UFP4_ERR_SHAPE;
+    const int64_t total = host_offsets[num_groups];
+    if (layout == UFP4_BWD_DW) {
+        // reduction grouped: A [N][total], B [Kout][total], C [num_groups * N][Kout]
+        if (A->k != total) return UFP4_ERR_SHAPE;
+        return ufp4::gemm_dispatch(A, B, C, ldc, c_is_bf16, path, 2, A->rows, B->rows, A->k, offsets, host_offsets,
+                                   num_groups, group_n, workspace, workspace_bytes, dev_status, stream);
+    }
+    // rows grouped: A [total][K], B [num_groups * group_n][K], C [total][group_n]
+    if (A->rows != total || group_n < 1 || B->rows != (int64_t)num_groups * group_n) return UFP4_ERR_SHAPE;
+    return ufp4::gemm_dispatch(A, B, C, ldc, c_is_bf16, path, 1, A->rows, group_n, A->k, offsets, host_offsets,
+                               num_groups, group_n, workspace, workspace_bytes, dev_status, stream);
+}

@@ -1,0 +1,114 @@
+"""The UFP4 linear-layer training step (Sec. 4, Table 1) assembled from the library's calls.
+
+One step of a linear layer Y = X W^T is: quantize X and W (RTNE) and dY (SR), each along both axes in one pass, then
+the three products fwd_y = X W^T, bwd_dx = dY W and bwd_dw = dY^T X, each on the pair of variants whose 16-blocks and
+RHT run along that product's reduction dimension (Sec. 2.2, last paragraph).  This module only sequences library
+calls and owns the buffers; all arithmetic is in libufp4's kernels.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as ufp4
+
+
+class Ufp4Linear:
+    """Preallocated buffers and the 3-quantize + 3-GEMM step for one dense layer (T tokens, K in, N out)."""
+
+    def __init__(self, tokens: int, in_features: int, out_features: int, device="cuda", grid: int = ufp4.GRID_INT4,
+                 scale_fmt: int = ufp4.SCALE_FP32, path: int = ufp4.PATH_AUTO, rht_block: int = 16,
+                 seed_rht: int = 1, seed_sr: int = 2, out_bf16: bool = False):
+        T, K, N = tokens, in_features, out_features
+        self.T, self.K, self.N = T, K, N
+        self.grid, self.scale_fmt, self.path, self.rht_block = grid, scale_fmt, path, rht_block
+        self.seed_rht, self.seed_sr = seed_rht, seed_sr
+        a = lambda r, k: ufp4.alloc_qtensor(r, k, grid, scale_fmt, device)
+        self.Xr, self.Xc = a(T, K), a(K, T)
+        self.Wr, self.Wc = a(N, K), a(K, N)
+        self.Gr, self.Gc = a(T, N), a(N, T)
+        dt = torch.bfloat16 if out_bf16 else torch.float32
+        self.Y = torch.empty(T, N, dtype=dt, device=device)
+        self.dX = torch.empty(T, K, dtype=dt, device=device)
+        self.dW = torch.empty(N, K, dtype=dt, device=device)
+        need = max(ufp4.gemm_workspace_bytes(self.Xr, self.Wr, path), ufp4.gemm_workspace_bytes(self.Gr, self.Wc, path),
+                   ufp4.gemm_workspace_bytes(self.Gc, self.Xc, path))
+        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    # number of kernel launches one call makes (for the benchmark's launch count)
+    launches_quantize = 3
+
+    def quantize(self, X, W, dY, stream=None):
+        kw = dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
+                  seed_rht=self.seed_rht, dev_status=self.dev_status, stream=stream)
+        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, **kw)
+        ufp4.quantize(W, rounding=ufp4.ROUND_RTNE, out_row=self.Wr, out_col=self.Wc, **kw)
+        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, **kw)
+
+    def gemms(self, stream=None):
+        kw = dict(path=self.path, workspace=self.workspace, dev_status=self.dev_status, stream=stream)
+        ufp4.gemm(self.Xr, self.Wr, out=self.Y, layout=ufp4.FWD_Y, **kw)
+        ufp4.gemm(self.Gr, self.Wc, out=self.dX, layout=ufp4.BWD_DX, **kw)
+        ufp4.gemm(self.Gc, self.Xc, out=self.dW, layout=ufp4.BWD_DW, **kw)
+
+    def step(self, X, W, dY, stream=None):
+        self.quantize(X, W, dY, stream)
+        self.gemms(stream)
+        return self.Y, self.dX, self.dW
+
+    @property
+    def flops(self) -> int:
+        return 3 * 2 * self.T * self.K * self.N
+
+    @property
+    def quantize_elements(self) -> int:
+        return self.T * self.K + self.N * self.K + self.T * self.N
+
+
+class Ufp4MoE:
+    """The same step for an MoE expert layer: rows of X / dY grouped by expert (offsets), weights [E][F][H]."""
+
+    def __init__(self, offsets_host: torch.Tensor, hidden: int, ffn: int, device="cuda", grid: int = ufp4.GRID_INT4,
+                 scale_fmt: int = ufp4.SCALE_FP32, path: int = ufp4.PATH_AUTO, rht_block: int = 16, seed_rht: int = 1,
+                 seed_sr: int = 2, out_bf16: bool = False):
+        self.offsets_host = offsets_host.to(torch.int64).contiguous()
+        self.offsets_dev = self.offsets_host.to(device)
+        E, R, H, F = offsets_host.numel() - 1, int(offsets_host[-1]), hidden, ffn
+        self.E, self.R, self.H, self.F = E, R, H, F
+        self.grid, self.scale_fmt, self.path, self.rht_block = grid, scale_fmt, path, rht_block
+        self.seed_rht, self.seed_sr = seed_rht, seed_sr
+        a = lambda r, k: ufp4.alloc_qtensor(r, k, grid, scale_fmt, device)
+        self.Xr, self.Xc = a(R, H), a(H, R)
+        self.Wr, self.Wc = a(E * F, H), a(E * H, F)
+        self.Gr, self.Gc = a(R, F), a(F, R)
+        dt = torch.bfloat16 if out_bf16 else torch.float32
+        self.Y = torch.empty(R, F, dtype=dt, device=device)
+        self.dX = torch.empty(R, H, dtype=dt, device=device)
+        self.dW = torch.empty(E * F, H, dtype=dt, device=device)
+        need = max(ufp4.gemm_workspace_bytes(self.Xr, self.Wr, path), ufp4.gemm_workspace_bytes(self.Gr, self.Wc, path),
+                   ufp4.gemm_workspace_bytes(self.Gc, self.Xc, path))
+        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def quantize(self, X, W, dY, stream=None):
+        kw = dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
+                  seed_rht=self.seed_rht, dev_status=self.dev_status, stream=stream)
+        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, **kw)
+        ufp4.quantize_batched(W.view(self.E, self.F, self.H), rounding=ufp4.ROUND_RTNE, out_row=self.Wr,
+                              out_col=self.Wc, **kw)
+        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, **kw)
+
+    def gemms(self, stream=None):
+        kw = dict(path=self.path, workspace=self.workspace, dev_status=self.dev_status, stream=stream)
+        ufp4.gemm_grouped(self.Xr, self.Wr, self.offsets_dev, self.offsets_host, self.F, ufp4.FWD_Y, out=self.Y, **kw)
+        ufp4.gemm_grouped(self.Gr, self.Wc, self.offsets_dev, self.offsets_host, self.H, ufp4.BWD_DX, out=self.dX, **kw)
+        ufp4.gemm_grouped(self.Gc, self.Xc, self.offsets_dev, self.offsets_host, self.F, ufp4.BWD_DW, out=self.dW, **kw)
+
+    def step(self, X, W, dY, stream=None):
+        self.quantize(X, W, dY, stream)
+        self.gemms(stream)
+        return self.Y, self.dX, self.dW
+
+    def flops(self, counts: torch.Tensor) -> int:
+        """Useful flops: unpadded routed rows only."""
+        return 3 * 2 * int(counts.sum()) * self.H * self.F

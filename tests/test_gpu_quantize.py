@@ -1,0 +1,150 @@
+"""Parity of the CUDA quantizer with the CPU oracle: codes, scales and SR draws bit-exact, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_qtensor_equal, oracle_quantize
+from paper_2606_20381_b200 import binding as ufp4
+from paper_2606_20381_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+GRIDS = [ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1]
+
+
+def run_both(x, axis, **kw):
+    """Quantize on the GPU (axis BOTH/ROW/COL) and with the oracle; compare every output."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ts = kw.get("tensor_scale")
+    row, col = ufp4.quantize(x.cuda(), axis=axis, dev_status=status, **kw)
+    okw = dict(kw)
+    if ts is not None:
+        okw["tensor_scale"] = float(ts)
+    if row is not None:
+        assert_qtensor_equal(row, oracle_quantize(x, oracle.AXIS_ROW, **okw), f"row variant {kw}")
+    if col is not None:
+        assert_qtensor_equal(col, oracle_quantize(x, oracle.AXIS_COL, **okw), f"col variant {kw}")
+    assert int(status.item()) == 0
+    return row, col
+
+
+def test_tiny_layer_recipe():
+    """The tiny single-layer check: UFP4 settings of Table 1 (RTNE for X and W, SR for dY, RHT 16, FP32 scales) and
+    the same with the E2M1 grid."""
+    X, W, dY = inputs.tiny_layer(0)
+    for grid in (ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1):
+        for t in (X, W):
+            run_both(t, ufp4.AXIS_BOTH, rht_block=16, grid=grid, rounding=ufp4.ROUND_RTNE, seed_rht=1)
+        run_both(dY, ufp4.AXIS_BOTH, rht_block=16, grid=grid, rounding=ufp4.ROUND_SR, seed_rht=1, seed_sr=2)
+
+
+@pytest.mark.parametrize("grid", GRIDS)
+@pytest.mark.parametrize("rounding", [ufp4.ROUND_RTNE, ufp4.ROUND_SR])
+@pytest.mark.parametrize("scale_fmt", [ufp4.SCALE_FP32, ufp4.SCALE_POW2, ufp4.SCALE_E4M3_TENSOR])
+@pytest.mark.parametrize("rht_block", [0, 16])
+def test_all_variants_on_a_ragged_multi_tile_matrix(grid, rounding, scale_fmt, rht_block):
+    x = inputs.spiky_normal(272, 400, seed=5)          # 3 x 4 tiles of 128 with ragged edges in both directions
+    kw = dict(rht_block=rht_block, grid=grid, rounding=rounding, scale_fmt=scale_fmt, seed_rht=3, seed_sr=11)
+    if scale_fmt == ufp4.SCALE_E4M3_TENSOR:
+        gmax = {ufp4.GRID_INT4: 7.0, ufp4.GRID_E1M2: 1.75, ufp4.GRID_E2M1: 6.0}[grid]
+        kw["tensor_scale"] = float(np.float32(4.0 * x.float().abs().max().item() / (gmax * 448.0)))
+    run_both(x, ufp4.AXIS_BOTH, **kw)
+
+
+@pytest.mark.parametrize("shape", [(16, 16), (128, 128), (16, 2048), (2048, 16), (144, 16), (1040, 1296)])
+def test_shapes(shape):
+    x = inputs.heavy_tailed_activations(shape[0], shape[1], seed=shape[0] + shape[1])
+    run_both(x, ufp4.AXIS_BOTH, rht_block=16, seed_rht=1)
+    run_both(x, ufp4.AXIS_BOTH, rht_block=16, rounding=ufp4.ROUND_SR, seed_rht=1, seed_sr=77)
+
+
+def test_single_axis_calls_and_odd_row_counts():
+    x = inputs.normal_bf16(37, 96, 1.0, seed=9)       # 37 rows: row variant only
+    run_both(x, ufp4.AXIS_ROW, rht_block=16, seed_rht=2)
+    x = inputs.normal_bf16(1, 16, 1.0, seed=10)
+    run_both(x, ufp4.AXIS_ROW, rht_block=16, seed_rht=2)
+    x = inputs.normal_bf16(160, 208, 1.0, seed=11)
+    run_both(x, ufp4.AXIS_COL, rht_block=16, seed_rht=2)
+    run_both(x, ufp4.AXIS_ROW, rht_block=0)
+    with pytest.raises(ufp4.Ufp4Error):
+        ufp4.quantize(inputs.normal_bf16(37, 96, 1.0, seed=9).cuda(), axis=ufp4.AXIS_BOTH)
+
+
+def test_strided_input_and_preallocated_padded_outputs():
+    base = inputs.normal_bf16(128, 512, 1.0, seed=12).cuda()
+    x = base[:, 64:64 + 208]                            # row pitch 512, start offset 128 bytes
+    row, col = ufp4.quantize(x, axis=ufp4.AXIS_BOTH, rht_block=16, seed_rht=4)
+    xc = x.contiguous()
+    assert_qtensor_equal(row, oracle_quantize(xc, oracle.AXIS_ROW, rht_block=16, seed_rht=4), "strided row")
+    assert_qtensor_equal(col, oracle_quantize(xc, oracle.AXIS_COL, rht_block=16, seed_rht=4), "strided col")
+    # caller-chosen pitches: the padding must stay untouched
+    out_row = ufp4.QTensor(torch.full((128, 128), 0xEE, dtype=torch.uint8, device="cuda"),
+                           torch.full((128, 20), -1.0, dtype=torch.float32, device="cuda"), ufp4.GRID_INT4,
+                           ufp4.SCALE_FP32, 208)
+    ufp4.quantize(x, axis=ufp4.AXIS_ROW, rht_block=16, seed_rht=4, out_row=out_row)
+    assert_qtensor_equal(ufp4.QTensor(out_row.codes, out_row.scales[:, :13], 0, 0, 208),
+                         oracle_quantize(xc, oracle.AXIS_ROW, rht_block=16, seed_rht=4), "padded row")
+    assert torch.all(out_row.codes[:, 104:] == 0xEE) and torch.all(out_row.scales[:, 13:] == -1.0)
+
+
+def test_degenerate_values():
+    x = torch.zeros(64, 64, dtype=torch.bfloat16)
+    run_both(x, ufp4.AXIS_BOTH, rht_block=16, seed_rht=1)
+    x[3, 5] = 1e-35                                      # below the 2^-100 threshold: still a zero block
+    x[40, 17] = -2.5e-3
+    x[41, 17] = 3e30
+    x[10, :16] = 1.0                                     # a constant block: the RHT concentrates it in one coordinate
+    run_both(x, ufp4.AXIS_BOTH, rht_block=16, seed_rht=1)
+    run_both(x, ufp4.AXIS_BOTH, rht_block=0, rounding=ufp4.ROUND_SR, seed_sr=5)
+    # every BF16 bit pattern that is finite, in one tensor (65280 finite patterns padded to 256 x 256 with zeros)
+    bits = np.arange(65536, dtype=np.uint16)
+    bits = bits[(bits & 0x7F80) != 0x7F80]
+    allv = np.zeros(65536, dtype=np.uint16)
+    allv[: bits.size] = bits
+    xa = torch.from_numpy(allv.reshape(256, 256).copy()).view(torch.bfloat16)
+    xa = torch.where(xa.float().abs() > 1e30, torch.zeros_like(xa), xa)   # stay inside the documented |x'| <= 2^120
+    for grid in GRIDS:
+        run_both(xa, ufp4.AXIS_BOTH, rht_block=0, grid=grid)
+        run_both(xa, ufp4.AXIS_BOTH, rht_block=16, grid=grid, seed_rht=6)
+
+
+def test_nonfinite_input_sets_the_status_bit():
+    x = inputs.normal_bf16(32, 32, 1.0, seed=13)
+    x[7, 9] = float("inf")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ufp4.quantize(x.cuda(), axis=ufp4.AXIS_BOTH, dev_status=status)
+    assert int(status.item()) & ufp4.DEV_NONFINITE
+    x[7, 9] = float("nan")
+    status.zero_()
+    ufp4.quantize(x.cuda(), axis=ufp4.AXIS_BOTH, rht_block=0, dev_status=status)
+    assert int(status.item()) & ufp4.DEV_NONFINITE
+
+
+def test_batched_weights_stack_along_rows():
+    E, N, K = 3, 48, 160
+    W = inputs.normal_bf16(E * N, K, 0.02, seed=14)
+    row, col = ufp4.quantize_batched(W.cuda().view(E, N, K), axis=ufp4.AXIS_BOTH, rht_block=16, seed_rht=8)
+    assert_qtensor_equal(row, oracle_quantize(W, oracle.AXIS_ROW, rht_block=16, seed_rht=8), "stacked row variant")
+    for e in range(E):
+        ref = oracle_quantize(W[e * N:(e + 1) * N], oracle.AXIS_COL, rht_block=16, seed_rht=8)
+        assert_qtensor_equal(col.row_slice(e * K, (e + 1) * K), ref, f"col variant of expert {e}")
+    with pytest.raises(ufp4.Ufp4Error):
+        ufp4.quantize_batched(W.cuda().view(E, N, K), rounding=ufp4.ROUND_SR)
+
+
+def test_repeated_runs_are_bit_identical():
+    x = inputs.heavy_tailed_activations(512, 768, seed=15).cuda()
+    a = ufp4.quantize(x, axis=ufp4.AXIS_BOTH, rounding=ufp4.ROUND_SR, seed_rht=1, seed_sr=2)
+    for _ in range(3):
+        b = ufp4.quantize(x, axis=ufp4.AXIS_BOTH, rounding=ufp4.ROUND_SR, seed_rht=1, seed_sr=2)
+        for p, q in zip(a, b):
+            assert torch.equal(p.codes, q.codes) and torch.equal(p.scales, q.scales)
+
+
+def test_dense_layer_full_size():
+    """Dense-1.5B-class up-projection tensors at full size (X 8192x2048, W 8192x2048, dY 8192x8192)."""
+    X, W, dY = inputs.dense_layer(8192, 2048, 8192, seed=1, device="cuda")
+    run_both(X.cpu(), ufp4.AXIS_BOTH, rht_block=16, seed_rht=1)
+    run_both(W.cpu(), ufp4.AXIS_BOTH, rht_block=16, seed_rht=1, scale_fmt=ufp4.SCALE_POW2)
+    run_both(dY.cpu(), ufp4.AXIS_BOTH, rht_block=16, rounding=ufp4.ROUND_SR, seed_rht=1, seed_sr=2)
