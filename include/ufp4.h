@@ -149,6 +149,11 @@ size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, i
  * scales only); blocks whose exponent lies outside a row's window set UFP4_DEV_EXP_WINDOW. */
 typedef enum { UFP4_PATH_AUTO = 0, UFP4_PATH_EXACT = 1, UFP4_PATH_TENSOR = 2 } ufp4_gemm_path;
 
+/* Which path ufp4_gemm would take for these operands and this request (UFP4_PATH_EXACT or UFP4_PATH_TENSOR, given a
+ * sufficient workspace), or a negative status.  *kernel_launches (optional, host) receives the number of kernels one
+ * such call enqueues. */
+int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B, int path, int *kernel_launches);
+
 /*
  * C[m][n] = sum_k a[m][k] * b[n][k], a = value(code) * scale (Sec. 2.2, Y^ = Q_G(XH') Q_G(WH')^T).
  *   A [M][K], B [N][K] quantized tensors with equal k; grids may differ

@@ -23,7 +23,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libufp4.so")
 
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_qtensor_bytes", "ufp4_quantize",
-           "ufp4_quantize_batched", "ufp4_gemm_workspace_bytes", "ufp4_gemm", "ufp4_gemm_grouped"]
+           "ufp4_quantize_batched", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped"]
 
 
 class _QTensorStruct(C.Structure):
@@ -59,6 +59,8 @@ def lib():
         L.ufp4_quantize_batched.argtypes = [vp, i64, i64, i64, i64, i64, i32, i32, i32, i32, i32, u64, u64, qp, qp, vp, vp]
         L.ufp4_gemm_workspace_bytes.restype = sz
         L.ufp4_gemm_workspace_bytes.argtypes = [qp, qp, i32]
+        L.ufp4_gemm_path_taken.restype = i32
+        L.ufp4_gemm_path_taken.argtypes = [qp, qp, i32, C.POINTER(i32)]
         L.ufp4_gemm.restype = i32
         L.ufp4_gemm.argtypes = [qp, qp, vp, i64, i32, i32, i32, vp, sz, vp, vp]
         L.ufp4_gemm_grouped.restype = i32
@@ -174,6 +176,23 @@ def quantize_batched(x: torch.Tensor, axis: int = AXIS_BOTH, rht_block: int = 16
 def gemm_workspace_bytes(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:
     sa, sb = A.struct(), B.struct()
     return int(lib().ufp4_gemm_workspace_bytes(C.byref(sa), C.byref(sb), path))
+
+
+def gemm_path_taken(A: QTensor, B: QTensor, path: int = PATH_AUTO):
+    """(path the library would take, kernels one call launches)."""
+    sa, sb, n = A.struct(), B.struct(), C.c_int(0)
+    rc = lib().ufp4_gemm_path_taken(C.byref(sa), C.byref(sb), path, C.byref(n))
+    if rc < 0:
+        raise Ufp4Error(rc)
+    return rc, n.value
+
+
+def gemm_launch_count(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:
+    return gemm_path_taken(A, B, path)[1]
+
+
+def gemm_path_name(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> str:
+    return {PATH_EXACT: "exact", PATH_TENSOR: "tensor"}[gemm_path_taken(A, B, path)[0]]
 
 
 def _workspace(A, B, path, workspace):

@@ -7,6 +7,7 @@ int gemm_exact_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
                       int64_t M, int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n,
                       void *stream);
 size_t gemm_tensor_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
+int gemm_tensor_kernel_launches();
 bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
 int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                        int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
@@ -77,6 +78,20 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     if (!A || !B || path == UFP4_PATH_EXACT) return 0;
     if (A->scale_fmt != UFP4_SCALE_POW2 || B->scale_fmt != UFP4_SCALE_POW2) return 0;
     return ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
+}
+
+extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B, int path, int *kernel_launches) {
+    int rc = ufp4::check_operand(A);
+    if (rc != UFP4_OK) return rc;
+    rc = ufp4::check_operand(B);
+    if (rc != UFP4_OK) return rc;
+    if (path < 0 || path > 2) return UFP4_ERR_ENUM;
+    if (A->k != B->k) return UFP4_ERR_SHAPE;
+    bool tensor_ok = ufp4::gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0);
+    if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
+    int taken = (path == UFP4_PATH_EXACT || !tensor_ok) ? UFP4_PATH_EXACT : UFP4_PATH_TENSOR;
+    if (kernel_launches) *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : ufp4::gemm_tensor_kernel_launches();
+    return taken;
 }
 
 extern "C" int ufp4_gemm(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int layout,
