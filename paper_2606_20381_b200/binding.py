@@ -195,6 +195,14 @@ def gemm_path_name(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> str:
     return {PATH_EXACT: "exact", PATH_TENSOR: "tensor"}[gemm_path_taken(A, B, path)[0]]
 
 
+def _alloc_out(rows: int, cols: int, bf16: bool, device) -> torch.Tensor:
+    """[rows][cols] output whose rows start on 16-byte boundaries (the row pitch is padded if cols is odd-sized)."""
+    per16 = 8 if bf16 else 4
+    ld = (cols + per16 - 1) // per16 * per16
+    buf = torch.empty(rows, ld, dtype=torch.bfloat16 if bf16 else torch.float32, device=device)
+    return buf[:, :cols]
+
+
 def _workspace(A, B, path, workspace):
     need = gemm_workspace_bytes(A, B, path)
     if workspace is None and need > 0:
@@ -207,7 +215,7 @@ def gemm(A: QTensor, B: QTensor, out: torch.Tensor | None = None, out_bf16: bool
          stream=None) -> torch.Tensor:
     """ufp4_gemm: C[m][n] = sum_k a[m][k] b[n][k] for quantized A [M][K], B [N][K]."""
     if out is None:
-        out = torch.empty(A.rows, B.rows, dtype=torch.bfloat16 if out_bf16 else torch.float32, device=A.codes.device)
+        out = _alloc_out(A.rows, B.rows, out_bf16, A.codes.device)
     assert out.is_cuda and out.stride(1) == 1
     workspace = _workspace(A, B, path, workspace)
     sa, sb = A.struct(), B.struct()
@@ -227,11 +235,10 @@ def gemm_grouped(A: QTensor, B: QTensor, offsets_dev: torch.Tensor, offsets_host
     assert (not offsets_host.is_cuda) and offsets_host.dtype == torch.int64 and offsets_host.is_contiguous()
     G = offsets_host.numel() - 1
     if out is None:
-        dt = torch.bfloat16 if out_bf16 else torch.float32
         if layout == BWD_DW:
-            out = torch.empty(G * A.rows, B.rows, dtype=dt, device=A.codes.device)
+            out = _alloc_out(G * A.rows, B.rows, out_bf16, A.codes.device)
         else:
-            out = torch.empty(A.rows, group_n, dtype=dt, device=A.codes.device)
+            out = _alloc_out(A.rows, group_n, out_bf16, A.codes.device)
     workspace = _workspace(A, B, path, workspace)
     sa, sb = A.struct(), B.struct()
     _check(lib().ufp4_gemm_grouped(C.byref(sa), C.byref(sb), out.data_ptr(), out.stride(0),

@@ -1,11 +1,518 @@
-// Placeholder until the tcgen05 path is wired in: reports itself unsupported so dispatch falls back to the exact path.
+// Tensor-core path of the block-scaled 4-bit GEMM (Sec. 2.2: Y^ = Q_G(XH') Q_G(WH')^T) for power-of-two block scales.
+//
+// B200's tensor cores have no uniform 4-bit element type (the paper's premise, Sec. 1 and Sec. 6), so the product is
+// computed exactly on 8-bit floating-point operands instead: with a power-of-two block scale 2^e, the dequantized
+// value q * 2^e (|q| <= 7, or 2*value <= 12 for the E2M1 grid: at most 3 significant bits) is exactly representable
+// in E5M2 once a per-row reference exponent is factored out.  Two kernels:
+//   1. decode_rows_kernel: packed nibbles + scales  ->  E5M2 bytes [rows][K] and one FP32 reference scale per row
+//      (caller's workspace); blocks more than 2^26 below the row's largest block are flushed and reported.
+//   2. gemm_tc_kernel: persistent, warp-specialised.  One thread issues TMA tile loads (128B-swizzled, 4-stage ring),
+//      one thread issues tcgen05.mma kind::f8f6f4 (M128 x N256 x K32) into a double-buffered FP32 accumulator in
+//      tensor memory, four warps drain accumulators with tcgen05.ld, apply refA[m] * refB[n] and store C.
+// Every products q_a 2^ea * q_b 2^eb is exact; accumulation is the tensor core's FP32.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
 #include "common.cuh"
+
 namespace ufp4 {
-size_t gemm_tensor_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
-int gemm_tensor_kernel_launches() { return 0; }
-bool gemm_tensor_supported(const ufp4_qtensor *, const ufp4_qtensor *, int64_t, int64_t, int64_t, int) { return false; }
-int gemm_tensor_launch(const ufp4_qtensor *, const ufp4_qtensor *, void *, int64_t, int, int, int64_t, int64_t, int64_t,
-                       const int64_t *, const int64_t *, int, int64_t, void *, size_t, int32_t *, void *) {
-    return UFP4_ERR_UNSUPPORTED;
+
+constexpr int kTM = 128, kTN = 256, kTK = 128;     // CTA tile (bytes along K: one E5M2 byte per element)
+constexpr int kStages = 4;
+constexpr int kUmmaK = 32;                          // K of one kind::f8f6f4 instruction
+constexpr int kAStage = kTM * kTK, kBStage = kTN * kTK;
+constexpr int kTcThreads = 192;                     // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-5: epilogue
+constexpr int kBarrierBytes = 256;
+constexpr int kTcSmem = kStages * (kAStage + kBStage) + kBarrierBytes + 1024;
+constexpr int kTmemCols = 512;
+constexpr int kDMax = 12, kDMin = -14;              // exponent window of a row, relative to its reference
+constexpr uint32_t kWaitLimit = 1u << 24;           // bounded mbarrier waits
+
+// ------------------------------------------------------------------------------------------------------------------
+// decode
+// ------------------------------------------------------------------------------------------------------------------
+
+struct DecodeParams {
+    const uint8_t *codes;
+    const float *scales;
+    int64_t ldc, lds, K;
+    int grid;
+    uint8_t *out8;      // [rows][K]
+    float *ref;         // [rows]
+    int32_t *dev_status;
+};
+
+__global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) {
+    __shared__ int red[8];
+    const int64_t row = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int64_t nkb = P.K >> 4;
+    const float *srow = P.scales + row * P.lds;
+
+    int emax = -1000;
+    for (int64_t kb = tid; kb < nkb; kb += 256) {
+        uint32_t b = __float_as_uint(srow[kb]);
+        if (b != 0u) emax = max(emax, (int)((b >> 23) & 0xFFu) - 127);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, o));
+    if ((tid & 31) == 0) red[tid >> 5] = emax;
+    __syncthreads();
+    emax = red[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) emax = max(emax, red[i]);
+    if (emax == -1000) emax = kDMax;                 // all-zero row
+    const int eref = emax - kDMax;
+    const float unit = P.grid == UFP4_GRID_INT4 ? 1.0f : (P.grid == UFP4_GRID_E1M2 ? 0.25f : 0.5f);
+    if (tid == 0) P.ref[row] = ldexpf(unit, eref);
+
+    bool flushed = false;
+    const uint8_t *crow = P.codes + row * P.ldc;
+    uint8_t *orow = P.out8 + row * P.K;
+    for (int64_t kb = tid; kb < nkb; kb += 256) {
+        uint32_t sb = __float_as_uint(srow[kb]);
+        uint2 cw = *reinterpret_cast<const uint2 *>(crow + kb * 8);
+        uint32_t out[4] = {0u, 0u, 0u, 0u};
+        int d = (int)((sb >> 23) & 0xFFu) - 127 - eref;
+        if (sb != 0u && d < kDMin) {
+            flushed |= (cw.x | cw.y) != 0u;
+        } else if (sb != 0u) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                uint32_t nib = ((j < 8 ? cw.x : cw.y) >> (4 * (j & 7))) & 0xFu;
+                uint32_t sign, mag;
+                if (P.grid == UFP4_GRID_INT4) {
+                    sign = nib >> 3;
+                    mag = sign ? (16u - nib) : nib;
+                } else {
+                    sign = nib >> 3;
+                    mag = nib & 7u;
+                    if (P.grid == UFP4_GRID_E2M1) mag = mag < 2u ? mag : (2u + (mag & 1u)) << ((mag >> 1) - 1u);
+                }
+                uint32_t byte = 0u;
+                if (mag) {
+                    // mag = 2^k (1 + f/4): E5M2 byte = sign | (15 + k + d) << 2 | f
+                    int k = 31 - __clz((int)mag);
+                    uint32_t f = ((mag << 2) >> k) & 3u;
+                    byte = (sign << 7) | ((uint32_t)(15 + k + d) << 2) | f;
+                }
+                out[j >> 2] |= byte << (8 * (j & 3));
+            }
+        }
+        *reinterpret_cast<uint4 *>(orow + kb * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+    if (flushed && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
 }
+
+// ------------------------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0u;
+}
+
+// Bounded wait: gives up after kWaitLimit polls or when another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 64u) {
+            if (*abort_flag) return false;
+            __nanosleep(32);
+        }
+    }
+    *abort_flag = 1u;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p; }"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major, 128B-swizzled shared-memory operand: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);          // start address
+    d |= (uint64_t)1u << 16;                          // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024u >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1u << 46;                          // descriptor version of this architecture
+    d |= (uint64_t)2u << 61;                          // 128-byte swizzle
+    return d;
+}
+
+// kind::f8f6f4, A = B = E5M2, D = F32, both K-major, M = 128, N = 256.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTN >> 3) << 17) | ((uint32_t)(kTM >> 4) << 24);
+
+// ------------------------------------------------------------------------------------------------------------------
+// GEMM
+// ------------------------------------------------------------------------------------------------------------------
+
+struct TcParams {
+    void *C;
+    int64_t ldc;
+    int c_is_bf16;
+    int64_t M, N, K;          // tile space M x N; K is the whole reduction length of the operands
+    int mode;                 // 0 plain, 1 rows grouped, 2 reduction grouped
+    const int64_t *offsets;
+    int num_groups;
+    int64_t group_n;
+    const float *refA, *refB;
+    int32_t *dev_status;
+    int mt, nt, total_tiles;
+};
+
+struct TileInfo {
+    int64_t m0, n0, b_row0, c_row0;
+    int kb0, nkb;
+};
+
+__device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile) {
+    TileInfo t;
+    const int per_group = P.mt * P.nt;
+    const int g = (P.mode == 2) ? tile / per_group : 0;
+    const int rem = tile - g * per_group;
+    t.m0 = (int64_t)(rem / P.nt) * kTM;
+    t.n0 = (int64_t)(rem % P.nt) * kTN;
+    t.b_row0 = 0;
+    t.c_row0 = 0;
+    t.kb0 = 0;
+    t.nkb = (int)((P.K + kTK - 1) / kTK);
+    if (P.mode == 1) {
+        int lo = 0, hi = P.num_groups;
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (P.offsets[mid] <= t.m0) lo = mid; else hi = mid;
+        }
+        t.b_row0 = (int64_t)lo * P.group_n;
+    } else if (P.mode == 2) {
+        t.kb0 = (int)(P.offsets[g] / kTK);
+        t.nkb = (int)((P.offsets[g + 1] - P.offsets[g]) / kTK);
+        t.c_row0 = (int64_t)g * P.M;
+    }
+    return t;
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *smem = smem_raw + (base - raw);
+    const uint32_t sA = base, sB = base + kStages * kAStage;
+    const uint32_t bars = base + kStages * (kAStage + kBStage);
+    const uint32_t full_bar = bars, empty_bar = bars + 8 * kStages;
+    const uint32_t tfull_bar = bars + 16 * kStages, tempty_bar = tfull_bar + 16;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kStages * (kAStage + kBStage) + 16 * kStages + 32);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar + 8 * a, 1);
+            mbar_init(tempty_bar + 8 * a, 4);
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- TMA producer
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+                const TileInfo t = tile_info(P, tile);
+                for (int kb = 0; kb < t.nkb; ++kb) {
+                    if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(full_bar + 8 * stage, kAStage + kBStage);
+                    const int32_t kc = (t.kb0 + kb) * kTK;
+                    tma_load_2d(sA + stage * kAStage, &tmA, kc, (int32_t)t.m0, full_bar + 8 * stage);
+                    tma_load_2d(sB + stage * kBStage, &tmB, kc, (int32_t)(t.b_row0 + t.n0), full_bar + 8 * stage);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+                const TileInfo t = tile_info(P, tile);
+                if (t.nkb == 0) continue;
+                if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * kTN;
+                for (int kb = 0; kb < t.nkb; ++kb) {
+                    if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t adesc = umma_desc_sw128(sA + stage * kAStage);
+                    const uint64_t bdesc = umma_desc_sw128(sB + stage * kBStage);
+#pragma unroll
+                    for (int k = 0; k < kTK / kUmmaK; ++k) {
+                        // advancing K inside the 128-byte swizzle span: +32 bytes = +2 in the (address >> 4) field
+                        tc_mma_f8(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kInstrDesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(empty_bar + 8 * stage);      // the stage is free once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                tc_commit(tfull_bar + 8 * acc);            // accumulator complete
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1u;
+            }
+        }
+    } else {
+        // ---------------- epilogue: TMEM -> registers -> scaled C
+        const int q = warp & 3;                            // TMEM lane quarter this warp may access
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+            const TileInfo t = tile_info(P, tile);
+            const int64_t m = t.m0 + q * 32 + lane;
+            const bool row_ok = m < P.M;
+            const float ra = row_ok ? P.refA[m] : 0.0f;
+            if (t.nkb > 0) {
+                if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+            }
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTN;
+#pragma unroll 1
+            for (int c = 0; c < kTN / 32; ++c) {
+                uint32_t v[32];
+                if (t.nkb > 0) {
+                    tc_ld32(taddr + (uint32_t)(c * 32), v);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                const int64_t n_base = t.n0 + c * 32;
+                if (row_ok && n_base < P.N) {
+                    const float *rb = P.refB + t.b_row0 + n_base;
+                    if (P.c_is_bf16) {
+                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(P.C) + (t.c_row0 + m) * P.ldc + n_base;
+                        if (n_base + 32 <= P.N) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                uint32_t pk[4];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    float lo = __uint_as_float(v[j + 2 * u]) * (ra * __ldg(rb + j + 2 * u));
+                                    float hi = __uint_as_float(v[j + 2 * u + 1]) * (ra * __ldg(rb + j + 2 * u + 1));
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+                                    pk[u] = *reinterpret_cast<uint32_t *>(&h);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            }
+                        } else {
+                            for (int j = 0; j < 32 && n_base + j < P.N; ++j)
+                                dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]) * (ra * __ldg(rb + j)));
+                        }
+                    } else {
+                        float *dst = static_cast<float *>(P.C) + (t.c_row0 + m) * P.ldc + n_base;
+                        if (n_base + 32 <= P.N) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                float4 o;
+                                o.x = __uint_as_float(v[j]) * (ra * __ldg(rb + j));
+                                o.y = __uint_as_float(v[j + 1]) * (ra * __ldg(rb + j + 1));
+                                o.z = __uint_as_float(v[j + 2]) * (ra * __ldg(rb + j + 2));
+                                o.w = __uint_as_float(v[j + 3]) * (ra * __ldg(rb + j + 3));
+                                *reinterpret_cast<float4 *>(dst + j) = o;
+                            }
+                        } else {
+                            for (int j = 0; j < 32 && n_base + j < P.N; ++j)
+                                dst[j] = __uint_as_float(v[j]) * (ra * __ldg(rb + j));
+                        }
+                    }
+                }
+            }
+            if (t.nkb > 0) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
+                acc ^= 1;
+                if (acc == 0) acc_phase ^= 1u;
+            }
+        }
+    }
+
+    // ---------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a bounded wait gave up: let any copy still in flight land before shared memory is released
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0 && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_WAIT_TIMEOUT);
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+static bool make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t K, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K};
+    cuuint32_t box[2] = {(cuuint32_t)kTK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+size_t gemm_tensor_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K) {
+    return round_up((size_t)a_rows * K, 256) + round_up((size_t)b_rows * K, 256) + round_up((size_t)a_rows * 4, 256) +
+           round_up((size_t)b_rows * 4, 256);
+}
+
+int gemm_tensor_kernel_launches() { return 3; }
+
+bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode) {
+    (void)mode;
+    if (A->scale_fmt != UFP4_SCALE_POW2 || B->scale_fmt != UFP4_SCALE_POW2) return false;
+    if (K % 16 != 0 || M < 1 || N < 1) return false;
+    if (A->rows > 0x7FFFFFFF || B->rows > 0x7FFFFFFF || K > 0x7FFFFFFF) return false;
+    return true;
+}
+
+int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
+                       int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
+                       int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                       void *stream) {
+    (void)host_offsets;
+    if (!aligned_to(workspace, 256)) return UFP4_ERR_ALIGN;
+    if (workspace_bytes < gemm_tensor_workspace_bytes(A->rows, B->rows, K)) return UFP4_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    uint8_t *A8 = ws;
+    uint8_t *B8 = A8 + round_up((size_t)A->rows * K, 256);
+    float *refA = reinterpret_cast<float *>(B8 + round_up((size_t)B->rows * K, 256));
+    float *refB = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(refA) + round_up((size_t)A->rows * 4, 256));
+
+    DecodeParams DA = {static_cast<const uint8_t *>(A->codes), static_cast<const float *>(A->scales), A->ld_codes_bytes,
+                       A->ld_scales, K, A->grid, A8, refA, dev_status};
+    DecodeParams DB = {static_cast<const uint8_t *>(B->codes), static_cast<const float *>(B->scales), B->ld_codes_bytes,
+                       B->ld_scales, K, B->grid, B8, refB, dev_status};
+    decode_rows_kernel<<<(unsigned)A->rows, 256, 0, st>>>(DA);
+    decode_rows_kernel<<<(unsigned)B->rows, 256, 0, st>>>(DB);
+    if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
+
+    CUtensorMap tmA, tmB;
+    if (!make_map(&tmA, A8, A->rows, K, kTM) || !make_map(&tmB, B8, B->rows, K, kTN)) return UFP4_ERR_CUDA;
+
+    TcParams P = {};
+    P.C = C; P.ldc = ldc; P.c_is_bf16 = c_is_bf16;
+    P.M = M; P.N = N; P.K = K; P.mode = mode;
+    P.offsets = offsets; P.num_groups = num_groups; P.group_n = group_n;
+    P.refA = refA; P.refB = refB; P.dev_status = dev_status;
+    P.mt = (int)((M + kTM - 1) / kTM);
+    P.nt = (int)((N + kTN - 1) / kTN);
+    const int64_t total = (int64_t)P.mt * P.nt * (mode == 2 ? num_groups : 1);
+    if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
+    P.total_tiles = (int)total;
+
+    static int num_sms = 0;
+    static bool attr_set = false;
+    if (!num_sms) {
+        int dev = 0;
+        UFP4_CUDA_OK(cudaGetDevice(&dev));
+        UFP4_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    }
+    if (!attr_set) {
+        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
+        attr_set = true;
+    }
+    const int grid = (int)(total < num_sms ? total : num_sms);
+    gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(tmA, tmB, P);
+    return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
+}
+
 }  // namespace ufp4

@@ -98,7 +98,7 @@ def test_gemm_rejects_bad_arguments_without_launching(lib):
     assert g(C.byref(A), C.byref(B), 0x4000, 32, 0, 0, 9, None, 0, None, None) == -4
     assert g(C.byref(_q(64, 120)), C.byref(_q(32, 120)), 0x4000, 32, 0, 0, 0, None, 0, None, None) == -2
     # the tensor-core path is only defined for power-of-two scales
-    assert g(C.byref(A), C.byref(B), 0x4000, 32, 0, 0, 2, None, 0, None, None) == -5
+    assert g(C.byref(A), C.byref(B), 0x4000, 32, 0, 0, 2, None, 0, None, None) == -5   # FP32 scales
     assert lib.ufp4_gemm_workspace_bytes(C.byref(A), C.byref(B), 1) == 0
 
 
