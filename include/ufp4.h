@@ -177,6 +177,29 @@ int ufp4_gemm_grouped(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
                       int path, const int64_t *offsets, const int64_t *host_offsets, int num_groups, int64_t group_n,
                       void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
+/*
+ * ufp4_gemm without any device allocation by anyone (the paper has no counterpart to this entry point; it exists for
+ * the library's users).  Some callers cannot provide the workspace ufp4_gemm's tensor-core path needs: a process
+ * whose device memory has all been handed to a framework's pool, or code running at a point where calling cudaMalloc
+ * is not allowed or would stall the whole device (it synchronises the device).  For them this call computes the same
+ * C[m][n] = sum_k a[m][k] * b[n][k] as ufp4_gemm(..., UFP4_PATH_TENSOR, ...) with its scratch (the decoded 8-bit
+ * operands and the per-row reference scales) in a fixed device array that is part of the library image.
+ *   - Limit: the scratch the shapes need, ufp4_gemm_workspace_bytes(A, B, UFP4_PATH_TENSOR), must not exceed
+ *     ufp4_gemm_noalloc_max_scratch_bytes() (16 MiB: e.g. A and B of 2048 rows each at K = 4096); beyond it the call
+ *     returns UFP4_ERR_WORKSPACE and launches nothing.  Every GPU that loads the library holds those 16 MiB until exit.
+ *   - Both operands must use UFP4_SCALE_POW2 (else UFP4_ERR_UNSUPPORTED).  C as in ufp4_gemm.
+ *   - The first call on each device looks up the array's device address (that device must be current); make that first
+ *     call outside any stream capture.  The call itself calls no cudaMalloc / cudaFree and no allocating library.
+ *   - All calls share the one array and it keeps the last call's contents; each call rewrites every byte it reads, so
+ *     nothing needs clearing, but two calls that overlap on the GPU (different streams, or different host threads)
+ *     race on it: serialise them on one stream.
+ */
+int ufp4_gemm_noalloc(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16,
+                      int32_t *dev_status, void *stream);
+
+/* Size in bytes of the fixed scratch array behind ufp4_gemm_noalloc. */
+size_t ufp4_gemm_noalloc_max_scratch_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libufp4.so")
 
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_qtensor_bytes", "ufp4_quantize",
-           "ufp4_quantize_batched", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped"]
+           "ufp4_quantize_batched", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
+           "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes"]
 
 
 class _QTensorStruct(C.Structure):
@@ -65,6 +66,10 @@ def lib():
         L.ufp4_gemm.argtypes = [qp, qp, vp, i64, i32, i32, i32, vp, sz, vp, vp]
         L.ufp4_gemm_grouped.restype = i32
         L.ufp4_gemm_grouped.argtypes = [qp, qp, vp, i64, i32, i32, i32, vp, vp, i32, i64, vp, sz, vp, vp]
+        L.ufp4_gemm_noalloc.restype = i32
+        L.ufp4_gemm_noalloc.argtypes = [qp, qp, vp, i64, i32, vp, vp]
+        L.ufp4_gemm_noalloc_max_scratch_bytes.restype = sz
+        L.ufp4_gemm_noalloc_max_scratch_bytes.argtypes = []
         _lib = L
     return _lib
 
@@ -246,5 +251,24 @@ def gemm_grouped(A: QTensor, B: QTensor, offsets_dev: torch.Tensor, offsets_host
                                    offsets_host.data_ptr(), G, group_n,
                                    workspace.data_ptr() if workspace is not None else None,
                                    workspace.numel() if workspace is not None else 0,
+                                   dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
+    return out
+
+
+def gemm_noalloc_max_scratch_bytes() -> int:
+    return int(lib().ufp4_gemm_noalloc_max_scratch_bytes())
+
+
+def gemm_noalloc(A: QTensor, B: QTensor, out: torch.Tensor, dev_status: torch.Tensor | None = None, stream=None):
+    """ufp4_gemm_noalloc: the tensor-core GEMM with its scratch in the library's fixed device array.
+
+    For callers that may not allocate device memory (all of it already belongs to a pool, or an allocation would stall
+    the device at this point): `out` must be preallocated by the caller, and this wrapper allocates nothing either.
+    Calls share one scratch array, so keep them on one stream.  Shapes whose scratch exceeds
+    gemm_noalloc_max_scratch_bytes() raise Ufp4Error (workspace)."""
+    assert out.is_cuda and out.stride(1) == 1
+    sa, sb = A.struct(), B.struct()
+    _check(lib().ufp4_gemm_noalloc(C.byref(sa), C.byref(sb), out.data_ptr(), out.stride(0),
+                                   int(out.dtype == torch.bfloat16),
                                    dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
     return out

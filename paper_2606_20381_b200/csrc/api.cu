@@ -8,6 +8,9 @@ int gemm_exact_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
                       void *stream);
 size_t gemm_tensor_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
 int gemm_tensor_kernel_launches();
+int gemm_noalloc_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16,
+                        int32_t *dev_status, void *stream);
+size_t gemm_noalloc_max_bytes();
 bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
 int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                        int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
@@ -131,4 +134,18 @@ extern "C" int ufp4_gemm_grouped(const ufp4_qtensor *A, const ufp4_qtensor *B, v
     if (A->rows != total || group_n < 1 || B->rows != (int64_t)num_groups * group_n) return UFP4_ERR_SHAPE;
     return ufp4::gemm_dispatch(A, B, C, ldc, c_is_bf16, path, 1, A->rows, group_n, A->k, offsets, host_offsets,
                                num_groups, group_n, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" size_t ufp4_gemm_noalloc_max_scratch_bytes(void) { return ufp4::gemm_noalloc_max_bytes(); }
+
+extern "C" int ufp4_gemm_noalloc(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16,
+                                 int32_t *dev_status, void *stream) {
+    int rc = ufp4::check_operand(A);
+    if (rc != UFP4_OK) return rc;
+    rc = ufp4::check_operand(B);
+    if (rc != UFP4_OK) return rc;
+    if (!C) return UFP4_ERR_NULL;
+    if (A->k != B->k || ldc < B->rows) return UFP4_ERR_SHAPE;
+    if (!ufp4::aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
+    return ufp4::gemm_noalloc_launch(A, B, C, ldc, c_is_bf16, dev_status, stream);
 }

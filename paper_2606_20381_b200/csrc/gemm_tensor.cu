@@ -515,4 +515,43 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------------------------------------------------------
+// Allocation-free variant of the tensor-core GEMM: its scratch lives in this file-scope device array, which every GPU
+// that loads the library holds until the process exits.
+// ------------------------------------------------------------------------------------------------------------------
+
+constexpr size_t kNoAllocScratchBytes = (size_t)16 << 20;
+static __device__ __align__(256) uint8_t g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void *g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device.  In host code the array's name is only a handle, not an
+// address a kernel could use, so the address is asked for once per device (with that device current) and cached.
+static int noalloc_scratch(void **out) {
+    int dev = 0;
+    UFP4_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return UFP4_ERR_UNSUPPORTED;
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        UFP4_CUDA_OK(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return UFP4_OK;
+}
+
+int gemm_noalloc_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16,
+                        int32_t *dev_status, void *stream) {
+    if (!gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0)) return UFP4_ERR_UNSUPPORTED;
+    if (gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) > kNoAllocScratchBytes) return UFP4_ERR_WORKSPACE;
+    void *scratch = nullptr;
+    int rc = noalloc_scratch(&scratch);
+    if (rc != UFP4_OK) return rc;
+    return gemm_tensor_launch(A, B, C, ldc, c_is_bf16, 0, A->rows, B->rows, A->k, nullptr, nullptr, 1, B->rows, scratch,
+                              kNoAllocScratchBytes, dev_status, stream);
+}
+
+size_t gemm_noalloc_max_bytes() { return kNoAllocScratchBytes; }
+
 }  // namespace ufp4
