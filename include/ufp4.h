@@ -140,6 +140,14 @@ int ufp4_quantize_batched(const void *x, int64_t batch, int64_t batch_stride, in
                           uint64_t seed_sr, const ufp4_qtensor *out_row, const ufp4_qtensor *out_col,
                           int32_t *dev_status, void *stream);
 
+/*
+ * Self-check of the quantizer's scale arithmetic (Sec. 2.1: s_B = amax / g_max and x_i / s_B).  The kernel evaluates
+ * amax / g and g / amax with short FMA sequences instead of the generic division; this call compares both sequences
+ * with the IEEE-754 division for every FP32 mantissa at eight exponents of the supported range and g in {7, 1.75, 6},
+ * and adds the number of differing results to *dev_mismatches (device int32, zeroed by the caller; expected 0).
+ */
+int ufp4_selftest_division(int32_t *dev_mismatches, void *stream);
+
 /* Workspace the GEMM calls need for these operands (0 for the exact path). */
 size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path);
 

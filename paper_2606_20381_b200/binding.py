@@ -23,7 +23,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libufp4.so")
 
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_qtensor_bytes", "ufp4_quantize",
-           "ufp4_quantize_batched", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
+           "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
            "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes"]
 
 
@@ -58,6 +58,8 @@ def lib():
         L.ufp4_quantize.argtypes = [vp, i64, i64, i64, i32, i32, i32, i32, i32, u64, u64, qp, qp, vp, vp]
         L.ufp4_quantize_batched.restype = i32
         L.ufp4_quantize_batched.argtypes = [vp, i64, i64, i64, i64, i64, i32, i32, i32, i32, i32, u64, u64, qp, qp, vp, vp]
+        L.ufp4_selftest_division.restype = i32
+        L.ufp4_selftest_division.argtypes = [vp, vp]
         L.ufp4_gemm_workspace_bytes.restype = sz
         L.ufp4_gemm_workspace_bytes.argtypes = [qp, qp, i32]
         L.ufp4_gemm_path_taken.restype = i32
@@ -176,6 +178,13 @@ def quantize_batched(x: torch.Tensor, axis: int = AXIS_BOTH, rht_block: int = 16
                                        C.byref(sc) if sc is not None else None,
                                        dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
     return (out_row if axis != AXIS_COL else None), (out_col if axis != AXIS_ROW else None)
+
+
+def selftest_division(stream=None) -> int:
+    """Number of FP32 inputs for which the quantizer's division shortcuts differ from the IEEE division (expected 0)."""
+    n = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().ufp4_selftest_division(n.data_ptr(), _stream_ptr(stream)))
+    return int(n.item())
 
 
 def gemm_workspace_bytes(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:

@@ -148,3 +148,8 @@ def test_dense_layer_full_size():
     run_both(X.cpu(), ufp4.AXIS_BOTH, rht_block=16, seed_rht=1)
     run_both(W.cpu(), ufp4.AXIS_BOTH, rht_block=16, seed_rht=1, scale_fmt=ufp4.SCALE_POW2)
     run_both(dY.cpu(), ufp4.AXIS_BOTH, rht_block=16, rounding=ufp4.ROUND_SR, seed_rht=1, seed_sr=2)
+
+
+def test_division_shortcuts_match_ieee_division_exhaustively():
+    """The kernel's amax / g and g / amax sequences against the IEEE division: all 2^23 mantissas x 8 exponents x 3 g."""
+    assert ufp4.selftest_division() == 0
