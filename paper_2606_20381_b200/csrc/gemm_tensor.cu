@@ -24,7 +24,14 @@ constexpr int kUmmaK = 32;                          // K of one kind::f8f6f4 ins
 constexpr int kAStage = kTM * kTK, kBStage = kTN * kTK;
 constexpr int kTcThreads = 192;                     // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-5: epilogue
 constexpr int kBarrierBytes = 256;
-constexpr int kTcSmem = kStages * (kAStage + kBStage) + kBarrierBytes + 1024;
+constexpr int kEpiBufBytes = 32 * 128;              // one staged 32-row x 32-column chunk (FP32; BF16 uses half of it)
+constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;     // four epilogue warps, double-buffered
+constexpr int kRefBBytes = 2 * kTN * 4;             // refB of the current and the next tile
+// layout: operand ring | epilogue staging | refB | barriers.  The dynamic shared-memory base is 1024-byte aligned.
+constexpr int kOffEpi = kStages * (kAStage + kBStage);
+constexpr int kOffRefB = kOffEpi + kEpiBytes;
+constexpr int kOffBars = kOffRefB + kRefBBytes;
+constexpr int kTcSmem = kOffBars + kBarrierBytes;
 constexpr int kTmemCols = 512;
 constexpr int kDMax = 12, kDMin = -14;              // exponent window of a row, relative to its reference
 
@@ -66,37 +73,38 @@ __global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) 
     const float unit = P.grid == UFP4_GRID_INT4 ? 1.0f : (P.grid == UFP4_GRID_E1M2 ? 0.25f : 0.5f);
     if (tid == 0) P.ref[row] = ldexpf(unit, eref);
 
+    // E5M2 bytes of the magnitudes 1..7 of a grid at d = 0, i.e. mag = 2^k (1 + f/4) -> (15 + k) << 2 | f; entry 0 is 0.
+    // Uniform grids: 1, 2, 3, 4, 5, 6, 7.  E2M1 (2 * value): 1, 2, 3, 4, 6, 8, 12.
+    const bool e2m1 = P.grid == UFP4_GRID_E2M1;
+    const uint32_t lut_lo0 = e2m1 ? 0x42403C00u : 0x42403C00u;      // entries 3, 2, 1, 0
+    const uint32_t lut_hi0 = e2m1 ? 0x4A484644u : 0x47464544u;      // entries 7, 6, 5, 4
     bool flushed = false;
     const uint8_t *crow = P.codes + row * P.ldc;
     uint8_t *orow = P.out8 + row * P.K;
     for (int64_t kb = tid; kb < nkb; kb += 256) {
-        uint32_t sb = __float_as_uint(srow[kb]);
-        uint2 cw = *reinterpret_cast<const uint2 *>(crow + kb * 8);
+        const uint32_t sb = __float_as_uint(srow[kb]);
+        const uint2 cw = *reinterpret_cast<const uint2 *>(crow + kb * 8);
         uint32_t out[4] = {0u, 0u, 0u, 0u};
-        int d = (int)((sb >> 23) & 0xFFu) - 127 - eref;
+        const int d = (int)((sb >> 23) & 0xFFu) - 127 - eref;
         if (sb != 0u && d < kDMin) {
             flushed |= (cw.x | cw.y) != 0u;
         } else if (sb != 0u) {
+            // per-block lookup table: the block's exponent offset is added to every non-zero entry
+            // (4 d is added to each byte; every byte stays inside [4, 0x7A], so the 32-bit wrap-around arithmetic below
+            // is an exact per-byte addition also for negative d)
+            const uint32_t off = (uint32_t)(d * 4);
+            const uint32_t lut_lo = lut_lo0 + off * 0x01010100u, lut_hi = lut_hi0 + off * 0x01010101u;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                uint32_t nib = ((j < 8 ? cw.x : cw.y) >> (4 * (j & 7))) & 0xFu;
-                uint32_t sign, mag;
-                if (P.grid == UFP4_GRID_INT4) {
-                    sign = nib >> 3;
-                    mag = sign ? (16u - nib) : nib;
-                } else {
-                    sign = nib >> 3;
-                    mag = nib & 7u;
-                    if (P.grid == UFP4_GRID_E2M1) mag = mag < 2u ? mag : (2u + (mag & 1u)) << ((mag >> 1) - 1u);
+            for (int h = 0; h < 2; ++h) {
+                uint32_t w = h ? cw.y : cw.x;
+                if (P.grid == UFP4_GRID_INT4) {             // two's complement -> sign | magnitude nibbles
+                    const uint32_t m = (w & 0x88888888u) >> 3;
+                    w = (w ^ (m * 7u)) + m;
                 }
-                uint32_t byte = 0u;
-                if (mag) {
-                    // mag = 2^k (1 + f/4): E5M2 byte = sign | (15 + k + d) << 2 | f
-                    int k = 31 - __clz((int)mag);
-                    uint32_t f = ((mag << 2) >> k) & 3u;
-                    byte = (sign << 7) | ((uint32_t)(15 + k + d) << 2) | f;
-                }
-                out[j >> 2] |= byte << (8 * (j & 3));
+                const uint32_t mag_lo = w & 0x7777u, mag_hi = (w >> 16) & 0x7777u;
+                const uint32_t sg_lo = (w >> 3) & 0x1111u, sg_hi = (w >> 19) & 0x1111u;
+                out[2 * h] = __byte_perm(lut_lo, lut_hi, mag_lo) | __byte_perm(0x00008000u, 0u, sg_lo);
+                out[2 * h + 1] = __byte_perm(lut_lo, lut_hi, mag_hi) | __byte_perm(0x00008000u, 0u, sg_hi);
             }
         }
         *reinterpret_cast<uint4 *>(orow + kb * 16) = make_uint4(out[0], out[1], out[2], out[3]);
@@ -160,6 +168,7 @@ struct TcParams {
     const float *refA, *refB;
     int32_t *dev_status;
     int mt, nt, total_tiles;
+    int n_unaligned;          // N * sizeof(element of C) is not a multiple of 16
 };
 
 struct TileInfo {
@@ -194,17 +203,17 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile) {
 }
 
 __global__ void __launch_bounds__(kTcThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams P) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t *smem = smem_raw + (base - raw);
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC, const TcParams P) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t base = smem_u32(smem);
     const uint32_t sA = base, sB = base + kStages * kAStage;
-    const uint32_t bars = base + kStages * (kAStage + kBStage);
+    const uint32_t bars = base + kOffBars;
     const uint32_t full_bar = bars, empty_bar = bars + 8 * kStages;
     const uint32_t tfull_bar = bars + 16 * kStages, tempty_bar = tfull_bar + 16;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kStages * (kAStage + kBStage) + 16 * kStages + 32);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kOffBars + 16 * kStages + 32);
     volatile uint32_t *abort_flag = tmem_slot + 1;
+    const uint32_t rb_bar = bars + 104;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -216,8 +225,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
             mbar_init(tempty_bar + 8 * a, 4);
+            mbar_init(rb_bar + 8 * a, 128);
         }
-        *abort_flag = 0u;
+        *abort_flag = (base & 1023u) ? 1u : 0u;      // the swizzled layouts below need the 1024-byte alignment
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -281,80 +291,122 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
         }
     } else {
-        // ---------------- epilogue: TMEM -> registers -> scaled C
+        // ---------------- epilogue: TMEM -> registers -> x refA[m] refB[n] -> swizzled shared staging -> TMA store of C
+        // A thread owns one accumulator row; per 32-column chunk it writes its 128 (FP32) or 64 (BF16) bytes into the
+        // warp's staging buffer in the 128B / 64B swizzle pattern and one lane hands the 32 x 32 box to the TMA, which
+        // clips rows >= M and columns >= N.  Staging is double-buffered so the next chunk is prepared while the
+        // previous box is still being read.
         const int q = warp & 3;                            // TMEM lane quarter this warp may access
-        int acc = 0;
-        uint32_t acc_phase = 0;
+        const int et = threadIdx.x - 64;                   // 0..127 among the epilogue threads
+        uint8_t *stage_base = smem + kOffEpi + q * 2 * kEpiBufBytes;
+        float *refb_s = reinterpret_cast<float *>(smem + kOffRefB);
+        const int g_tiles = P.mt * P.nt;
+        int acc = 0, sbuf = 0, rbuf = 0;
+        uint32_t acc_phase = 0, rb_phase[2] = {0u, 0u};
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
             const TileInfo t = tile_info(P, tile);
-            const int64_t m = t.m0 + q * 32 + lane;
-            const bool row_ok = m < P.M;
-            const float ra = row_ok ? P.refA[m] : 0.0f;
+            const int64_t m_own = t.m0 + q * 32 + lane;
+            const float ra = m_own < P.M ? P.refA[m_own] : 0.0f;
+            // refB of this tile's 256 columns into shared memory (two values per thread), double-buffered across tiles
+            {
+                float *dst = refb_s + rbuf * kTN;
+                const int64_t n = t.n0 + 2 * et;
+                dst[2 * et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
+                dst[2 * et + 1] = n + 1 < P.N ? P.refB[t.b_row0 + n + 1] : 0.0f;
+                // all 128 epilogue threads have written their two values (bounded, abortable wait instead of bar.sync)
+                mbar_arrive(rb_bar + 8 * rbuf);
+                if (!mbar_wait(rb_bar + 8 * rbuf, rb_phase[rbuf], abort_flag)) { ok = false; break; }
+                rb_phase[rbuf] ^= 1u;
+            }
+            const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s + rbuf * kTN);
+            rbuf ^= 1;
             if (t.nkb > 0) {
                 if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTN;
-#pragma unroll 1
+            const int32_t c_row = (int32_t)(t.m0 + q * 32), c_grp = (int32_t)(t.c_row0 / (P.M > 0 ? P.M : 1));
+            uint32_t v[2][32];
+            if (t.nkb > 0) tc_ld32(taddr, v[0]);
+#pragma unroll
             for (int c = 0; c < kTN / 32; ++c) {
-                uint32_t v[32];
+                const int cur = c & 1;
                 if (t.nkb > 0) {
-                    tc_ld32(taddr + (uint32_t)(c * 32), v);
                     tc_wait_ld();
+                    if (c + 1 < kTN / 32) tc_ld32(taddr + (uint32_t)((c + 1) * 32), v[cur ^ 1]);
+                    else {
+                        // every column of this accumulator has been read: hand it back to the MMA warp
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
+                    }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                    for (int j = 0; j < 32; ++j) v[cur][j] = 0u;
                 }
                 const int64_t n_base = t.n0 + c * 32;
-                if (row_ok && n_base < P.N) {
-                    const float *rb = P.refB + t.b_row0 + n_base;
-                    if (P.c_is_bf16) {
-                        __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(P.C) + (t.c_row0 + m) * P.ldc + n_base;
-                        if (n_base + 32 <= P.N) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                uint32_t pk[4];
-#pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    float lo = __uint_as_float(v[j + 2 * u]) * (ra * __ldg(rb + j + 2 * u));
-                                    float hi = __uint_as_float(v[j + 2 * u + 1]) * (ra * __ldg(rb + j + 2 * u + 1));
-                                    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-                                    pk[u] = *reinterpret_cast<uint32_t *>(&h);
-                                }
-                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                            }
-                        } else {
-                            for (int j = 0; j < 32 && n_base + j < P.N; ++j)
-                                dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]) * (ra * __ldg(rb + j)));
-                        }
-                    } else {
-                        float *dst = static_cast<float *>(P.C) + (t.c_row0 + m) * P.ldc + n_base;
-                        if (n_base + 32 <= P.N) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                float4 o;
-                                o.x = __uint_as_float(v[j]) * (ra * __ldg(rb + j));
-                                o.y = __uint_as_float(v[j + 1]) * (ra * __ldg(rb + j + 1));
-                                o.z = __uint_as_float(v[j + 2]) * (ra * __ldg(rb + j + 2));
-                                o.w = __uint_as_float(v[j + 3]) * (ra * __ldg(rb + j + 3));
-                                *reinterpret_cast<float4 *>(dst + j) = o;
-                            }
-                        } else {
-                            for (int j = 0; j < 32 && n_base + j < P.N; ++j)
-                                dst[j] = __uint_as_float(v[j]) * (ra * __ldg(rb + j));
+                if (n_base >= P.N || c_row >= P.M) continue;     // warp-uniform: the whole box would be clipped
+                if (n_base + 32 > P.N && P.n_unaligned) {
+                    // The TMA clips in 16-byte units: a last chunk whose valid part does not end on a 16-byte boundary
+                    // is written with plain predicated stores so that nothing right of column N is touched.
+                    if (m_own < P.M) {
+                        for (int j = 0; j < 32 && n_base + j < P.N; ++j) {
+                            const float val = __uint_as_float(v[cur][j]) * ra * refb_s[(rbuf ^ 1) * kTN + c * 32 + j];
+                            const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
+                            if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(val);
+                            else static_cast<float *>(P.C)[idx] = val;
                         }
                     }
+                    continue;
                 }
+                // the buffer used two chunks ago must have been read by its TMA store
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
+                uint8_t *buf = stage_base + sbuf * kEpiBufBytes;
+                if (P.c_is_bf16) {
+                    // 64-byte rows, 64B swizzle: 16-byte piece j of row r sits at piece j ^ ((r >> 1) & 3)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float4 r0 = rb4[c * 8 + 2 * j], r1 = rb4[c * 8 + 2 * j + 1];
+                        const uint32_t *x = &v[cur][8 * j];
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(x[0]) * ra * r0.x, __uint_as_float(x[1]) * ra * r0.y);
+                        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(x[2]) * ra * r0.z, __uint_as_float(x[3]) * ra * r0.w);
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(x[4]) * ra * r1.x, __uint_as_float(x[5]) * ra * r1.y);
+                        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(x[6]) * ra * r1.z, __uint_as_float(x[7]) * ra * r1.w);
+                        *reinterpret_cast<uint4 *>(buf + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) =
+                            make_uint4(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1),
+                                       *reinterpret_cast<uint32_t *>(&h2), *reinterpret_cast<uint32_t *>(&h3));
+                    }
+                } else {
+                    // 128-byte rows, 128B swizzle: 16-byte piece j of row r sits at piece j ^ (r & 7)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float4 r = rb4[c * 8 + j];
+                        const uint32_t *x = &v[cur][4 * j];
+                        *reinterpret_cast<float4 *>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                            make_float4(__uint_as_float(x[0]) * ra * r.x, __uint_as_float(x[1]) * ra * r.y,
+                                        __uint_as_float(x[2]) * ra * r.z, __uint_as_float(x[3]) * ra * r.w);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    asm volatile(
+                        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                        ::"l"(&tmC), "r"((int32_t)n_base), "r"(c_row), "r"(c_grp), "r"(smem_u32(buf)) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                sbuf ^= 1;
             }
             if (t.nkb > 0) {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1u;
             }
         }
+        (void)g_tiles;
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all C boxes written
+        __syncwarp();
     }
 
     // ---------------- teardown
@@ -430,6 +482,23 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     CUtensorMap tmA, tmB;
     if (!make_map(&tmA, A8, A->rows, K, kTM) || !make_map(&tmB, B8, B->rows, K, kTN)) return UFP4_ERR_CUDA;
 
+    // C as [groups][rows][cols] so that the TMA store clips at the end of each group's rows and at N
+    CUtensorMap tmC;
+    {
+        EncodeTiledFn fn = encode_tiled_fn();
+        if (!fn) return UFP4_ERR_CUDA;
+        const int64_t groups = mode == 2 ? num_groups : 1;
+        const cuuint64_t es = c_is_bf16 ? 2 : 4;
+        cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)groups};
+        cuuint64_t strides[2] = {(cuuint64_t)ldc * es, (cuuint64_t)M * (cuuint64_t)ldc * es};
+        cuuint32_t box[3] = {32, 32, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        if (fn(&tmC, c_is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, C, dims, strides, box,
+               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, c_is_bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return UFP4_ERR_CUDA;
+    }
+
     TcParams P = {};
     P.C = C; P.ldc = ldc; P.c_is_bf16 = c_is_bf16;
     P.M = M; P.N = N; P.K = K; P.mode = mode;
@@ -440,6 +509,7 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     const int64_t total = (int64_t)P.mt * P.nt * (mode == 2 ? num_groups : 1);
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     P.total_tiles = (int)total;
+    P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
 
     static int num_sms = 0;
     static bool attr_set = false;
@@ -453,7 +523,7 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
         attr_set = true;
     }
     const int grid = (int)(total < num_sms ? total : num_sms);
-    gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(tmA, tmB, P);
+    gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(tmA, tmB, tmC, P);
     return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 
