@@ -39,49 +39,54 @@ constexpr int kDMax = 12, kDMin = -14;              // exponent window of a row,
 // decode
 // ------------------------------------------------------------------------------------------------------------------
 
-struct DecodeParams {
+struct DecodeOperand {
     const uint8_t *codes;
     const float *scales;
-    int64_t ldc, lds, K;
+    int64_t ldc, lds, rows;
     int grid;
     uint8_t *out8;      // [rows][K]
     float *ref;         // [rows]
+};
+
+struct DecodeParams {
+    DecodeOperand op[2];    // A and B in one launch
+    int64_t K;
+    int64_t a_ctas;         // CTAs [0, a_ctas) work on A, the rest on B
     int32_t *dev_status;
 };
 
-__global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) {
-    __shared__ int red[8];
-    const int64_t row = blockIdx.x;
-    const int tid = threadIdx.x;
-    const int64_t nkb = P.K >> 4;
-    const float *srow = P.scales + row * P.lds;
+constexpr int kDecodeRowsPerCta = 8;   // one warp per row
 
+__global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) {
+    const bool is_b = (int64_t)blockIdx.x >= P.a_ctas;
+    const DecodeOperand &O = P.op[is_b ? 1 : 0];
+    const int lane = threadIdx.x & 31;
+    const int64_t row = ((int64_t)blockIdx.x - (is_b ? P.a_ctas : 0)) * kDecodeRowsPerCta + (threadIdx.x >> 5);
+    if (row >= O.rows) return;
+    const int64_t nkb = P.K >> 4;
+    const float *srow = O.scales + row * O.lds;
+
+    // largest block exponent of the row (power-of-two scales: the exponent field is the scale)
     int emax = -1000;
-    for (int64_t kb = tid; kb < nkb; kb += 256) {
-        uint32_t b = __float_as_uint(srow[kb]);
+    for (int64_t kb = lane; kb < nkb; kb += 32) {
+        const uint32_t b = __float_as_uint(srow[kb]);
         if (b != 0u) emax = max(emax, (int)((b >> 23) & 0xFFu) - 127);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, o));
-    if ((tid & 31) == 0) red[tid >> 5] = emax;
-    __syncthreads();
-    emax = red[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) emax = max(emax, red[i]);
     if (emax == -1000) emax = kDMax;                 // all-zero row
     const int eref = emax - kDMax;
-    const float unit = P.grid == UFP4_GRID_INT4 ? 1.0f : (P.grid == UFP4_GRID_E1M2 ? 0.25f : 0.5f);
-    if (tid == 0) P.ref[row] = ldexpf(unit, eref);
+    const float unit = O.grid == UFP4_GRID_INT4 ? 1.0f : (O.grid == UFP4_GRID_E1M2 ? 0.25f : 0.5f);
+    if (lane == 0) O.ref[row] = ldexpf(unit, eref);
 
     // E5M2 bytes of the magnitudes 1..7 of a grid at d = 0, i.e. mag = 2^k (1 + f/4) -> (15 + k) << 2 | f; entry 0 is 0.
     // Uniform grids: 1, 2, 3, 4, 5, 6, 7.  E2M1 (2 * value): 1, 2, 3, 4, 6, 8, 12.
-    const bool e2m1 = P.grid == UFP4_GRID_E2M1;
-    const uint32_t lut_lo0 = e2m1 ? 0x42403C00u : 0x42403C00u;      // entries 3, 2, 1, 0
-    const uint32_t lut_hi0 = e2m1 ? 0x4A484644u : 0x47464544u;      // entries 7, 6, 5, 4
+    const uint32_t lut_lo0 = 0x42403C00u;                                           // entries 3, 2, 1, 0
+    const uint32_t lut_hi0 = O.grid == UFP4_GRID_E2M1 ? 0x4A484644u : 0x47464544u;  // entries 7, 6, 5, 4
     bool flushed = false;
-    const uint8_t *crow = P.codes + row * P.ldc;
-    uint8_t *orow = P.out8 + row * P.K;
-    for (int64_t kb = tid; kb < nkb; kb += 256) {
+    const uint8_t *crow = O.codes + row * O.ldc;
+    uint8_t *orow = O.out8 + row * P.K;
+    for (int64_t kb = lane; kb < nkb; kb += 32) {
         const uint32_t sb = __float_as_uint(srow[kb]);
         const uint2 cw = *reinterpret_cast<const uint2 *>(crow + kb * 8);
         uint32_t out[4] = {0u, 0u, 0u, 0u};
@@ -89,15 +94,14 @@ __global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) 
         if (sb != 0u && d < kDMin) {
             flushed |= (cw.x | cw.y) != 0u;
         } else if (sb != 0u) {
-            // per-block lookup table: the block's exponent offset is added to every non-zero entry
-            // (4 d is added to each byte; every byte stays inside [4, 0x7A], so the 32-bit wrap-around arithmetic below
-            // is an exact per-byte addition also for negative d)
+            // per-block lookup table: 4 d is added to each non-zero entry; every byte stays inside [4, 0x7A], so the
+            // 32-bit wrap-around arithmetic below is an exact per-byte addition also for negative d
             const uint32_t off = (uint32_t)(d * 4);
             const uint32_t lut_lo = lut_lo0 + off * 0x01010100u, lut_hi = lut_hi0 + off * 0x01010101u;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t w = h ? cw.y : cw.x;
-                if (P.grid == UFP4_GRID_INT4) {             // two's complement -> sign | magnitude nibbles
+                if (O.grid == UFP4_GRID_INT4) {             // two's complement -> sign | magnitude nibbles
                     const uint32_t m = (w & 0x88888888u) >> 3;
                     w = (w ^ (m * 7u)) + m;
                 }
@@ -447,7 +451,7 @@ size_t gemm_tensor_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K) {
            round_up((size_t)b_rows * 4, 256);
 }
 
-int gemm_tensor_kernel_launches() { return 3; }
+int gemm_tensor_kernel_launches() { return 2; }
 
 bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode) {
     (void)mode;
@@ -471,12 +475,17 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     float *refA = reinterpret_cast<float *>(B8 + round_up((size_t)B->rows * K, 256));
     float *refB = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(refA) + round_up((size_t)A->rows * 4, 256));
 
-    DecodeParams DA = {static_cast<const uint8_t *>(A->codes), static_cast<const float *>(A->scales), A->ld_codes_bytes,
-                       A->ld_scales, K, A->grid, A8, refA, dev_status};
-    DecodeParams DB = {static_cast<const uint8_t *>(B->codes), static_cast<const float *>(B->scales), B->ld_codes_bytes,
-                       B->ld_scales, K, B->grid, B8, refB, dev_status};
-    decode_rows_kernel<<<(unsigned)A->rows, 256, 0, st>>>(DA);
-    decode_rows_kernel<<<(unsigned)B->rows, 256, 0, st>>>(DB);
+    DecodeParams D = {};
+    D.op[0] = DecodeOperand{static_cast<const uint8_t *>(A->codes), static_cast<const float *>(A->scales),
+                            A->ld_codes_bytes, A->ld_scales, A->rows, A->grid, A8, refA};
+    D.op[1] = DecodeOperand{static_cast<const uint8_t *>(B->codes), static_cast<const float *>(B->scales),
+                            B->ld_codes_bytes, B->ld_scales, B->rows, B->grid, B8, refB};
+    D.K = K;
+    D.a_ctas = (A->rows + kDecodeRowsPerCta - 1) / kDecodeRowsPerCta;
+    D.dev_status = dev_status;
+    const int64_t decode_ctas = D.a_ctas + (B->rows + kDecodeRowsPerCta - 1) / kDecodeRowsPerCta;
+    if (decode_ctas > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
+    decode_rows_kernel<<<(unsigned)decode_ctas, 256, 0, st>>>(D);
     if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
 
     CUtensorMap tmA, tmB;
