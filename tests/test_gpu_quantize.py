@@ -153,3 +153,25 @@ def test_dense_layer_full_size():
 def test_division_shortcuts_match_ieee_division_exhaustively():
     """The kernel's amax / g and g / amax sequences against the IEEE division: all 2^23 mantissas x 8 exponents x 3 g."""
     assert ufp4.selftest_division() == 0
+
+
+def test_per_bin_bias_measurement_agrees_with_the_oracle():
+    """The Shrinkage-Bias measurement used by the quantizer sweep (torch ops on the CUDA quantizer's output) against the
+    oracle's per-bin bias on the same tensor: the uniform grid is unbiased on interior levels, E2M1 is not."""
+    from paper_2606_20381_b200 import diagnostics
+    x = inputs.spiky_normal(512, 1024, seed=3)
+    for grid in (ufp4.GRID_INT4, ufp4.GRID_E2M1):
+        for rht in (0, 16):
+            row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=rht, grid=grid, seed_rht=1)
+            count, bias = diagnostics.per_bin_bias(x.cuda(), row, rht, 1)
+            ref = oracle_quantize(x, oracle.AXIS_ROW, rht_block=rht, grid=grid, seed_rht=1, want_y=True)
+            rc, rb = oracle.bin_bias(ref.y, ref.codes, grid)
+            assert np.array_equal(count.numpy(), rc)
+            assert np.allclose(bias.numpy(), rb, atol=2e-5, equal_nan=True)
+    # direction of the effect the paper describes: after RHT the E2M1 levels 2 and 4 shrink, the uniform grid does not
+    row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_E2M1, seed_rht=1)
+    _, b = diagnostics.per_bin_bias(x.cuda(), row, 16, 1)
+    assert b[4] < -0.05 and b[6] < -0.1
+    row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_INT4, seed_rht=1)
+    _, b = diagnostics.per_bin_bias(x.cuda(), row, 16, 1)
+    assert abs(b[1:7]).max() < 0.05     # what remains is the decreasing density inside symmetric bins, not geometry
