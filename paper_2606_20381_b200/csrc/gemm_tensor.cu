@@ -22,10 +22,11 @@ constexpr int kTM = 128, kTN = 256, kTK = 128;     // CTA tile (bytes along K: o
 constexpr int kStages = 4;
 constexpr int kUmmaK = 32;                          // K of one kind::f8f6f4 instruction
 constexpr int kAStage = kTM * kTK, kBStage = kTN * kTK;
-constexpr int kTcThreads = 192;                     // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-5: epilogue
+constexpr int kEpiWarps = 8;                        // two per TMEM lane quarter, each taking half of the columns
+constexpr int kTcThreads = 64 + 32 * kEpiWarps;      // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-9: epilogue
 constexpr int kBarrierBytes = 256;
 constexpr int kEpiBufBytes = 32 * 128;              // one staged 32-row x 32-column chunk (FP32; BF16 uses half of it)
-constexpr int kEpiBytes = 4 * 2 * kEpiBufBytes;     // four epilogue warps, double-buffered
+constexpr int kEpiBytes = kEpiWarps * kEpiBufBytes;  // one staging buffer per epilogue warp
 constexpr int kRefBBytes = 2 * kTN * 4;             // refB of the current and the next tile
 // layout: operand ring | epilogue staging | refB | barriers.  The dynamic shared-memory base is 1024-byte aligned.
 constexpr int kOffEpi = kStages * (kAStage + kBStage);
@@ -228,8 +229,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
-            mbar_init(tempty_bar + 8 * a, 4);
-            mbar_init(rb_bar + 8 * a, 128);
+            mbar_init(tempty_bar + 8 * a, kEpiWarps);
+            mbar_init(rb_bar + 8 * a, 32 * kEpiWarps);
         }
         *abort_flag = (base & 1023u) ? 1u : 0u;      // the swizzled layouts below need the 1024-byte alignment
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -301,24 +302,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // clips rows >= M and columns >= N.  Staging is double-buffered so the next chunk is prepared while the
         // previous box is still being read.
         const int q = warp & 3;                            // TMEM lane quarter this warp may access
-        const int et = threadIdx.x - 64;                   // 0..127 among the epilogue threads
-        uint8_t *stage_base = smem + kOffEpi + q * 2 * kEpiBufBytes;
+        const int half = (warp - 2) >> 2;                  // which four of the eight 32-column chunks this warp drains
+        const int et = threadIdx.x - 64;                   // 0..255 among the epilogue threads
+        uint8_t *buf = smem + kOffEpi + (warp - 2) * kEpiBufBytes;
         float *refb_s = reinterpret_cast<float *>(smem + kOffRefB);
-        const int g_tiles = P.mt * P.nt;
-        int acc = 0, sbuf = 0, rbuf = 0;
+        int acc = 0, rbuf = 0;
         uint32_t acc_phase = 0, rb_phase[2] = {0u, 0u};
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
             const TileInfo t = tile_info(P, tile);
             const int64_t m_own = t.m0 + q * 32 + lane;
             const float ra = m_own < P.M ? P.refA[m_own] : 0.0f;
-            // refB of this tile's 256 columns into shared memory (two values per thread), double-buffered across tiles
+            // refB of this tile's 256 columns into shared memory (one value per thread), double-buffered across tiles
             {
-                float *dst = refb_s + rbuf * kTN;
-                const int64_t n = t.n0 + 2 * et;
-                dst[2 * et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
-                dst[2 * et + 1] = n + 1 < P.N ? P.refB[t.b_row0 + n + 1] : 0.0f;
-                // all 128 epilogue threads have written their two values (bounded, abortable wait instead of bar.sync)
+                const int64_t n = t.n0 + et;
+                refb_s[rbuf * kTN + et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
+                // all epilogue threads have written their value (bounded, abortable wait instead of bar.sync)
                 mbar_arrive(rb_bar + 8 * rbuf);
                 if (!mbar_wait(rb_bar + 8 * rbuf, rb_phase[rbuf], abort_flag)) { ok = false; break; }
                 rb_phase[rbuf] ^= 1u;
@@ -332,13 +331,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTN;
             const int32_t c_row = (int32_t)(t.m0 + q * 32), c_grp = (int32_t)(t.c_row0 / (P.M > 0 ? P.M : 1));
             uint32_t v[2][32];
-            if (t.nkb > 0) tc_ld32(taddr, v[0]);
+            const int c_begin = 4 * half;
+            if (t.nkb > 0) tc_ld32(taddr + (uint32_t)(c_begin * 32), v[0]);
 #pragma unroll
-            for (int c = 0; c < kTN / 32; ++c) {
-                const int cur = c & 1;
+            for (int cc = 0; cc < 4; ++cc) {
+                const int c = c_begin + cc, cur = cc & 1;
                 if (t.nkb > 0) {
                     tc_wait_ld();
-                    if (c + 1 < kTN / 32) tc_ld32(taddr + (uint32_t)((c + 1) * 32), v[cur ^ 1]);
+                    if (cc + 1 < 4) tc_ld32(taddr + (uint32_t)((c + 1) * 32), v[cur ^ 1]);
                     else {
                         // every column of this accumulator has been read: hand it back to the MMA warp
                         tc_fence_before();
@@ -364,10 +364,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     continue;
                 }
-                // the buffer used two chunks ago must have been read by its TMA store
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                // the previous box must have been read out of the staging buffer by its TMA store
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 __syncwarp();
-                uint8_t *buf = stage_base + sbuf * kEpiBufBytes;
                 if (P.c_is_bf16) {
                     // 64-byte rows, 64B swizzle: 16-byte piece j of row r sits at piece j ^ ((r >> 1) & 3)
 #pragma unroll
@@ -401,14 +400,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         ::"l"(&tmC), "r"((int32_t)n_base), "r"(c_row), "r"(c_grp), "r"(smem_u32(buf)) : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
-                sbuf ^= 1;
             }
             if (t.nkb > 0) {
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1u;
             }
         }
-        (void)g_tiles;
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all C boxes written
         __syncwarp();
     }
