@@ -12,24 +12,36 @@
 // Every products q_a 2^ea * q_b 2^eb is exact; accumulation is the tensor core's FP32.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace ufp4 {
 
-constexpr int kTM = 128, kTN = 256, kTK = 128;     // CTA tile (bytes along K: one E5M2 byte per element)
-constexpr int kStages = 4;
+constexpr int kTM = 128, kTN = 256, kTK = 128;     // per-CTA output tile (bytes along K: one E5M2 byte per element)
 constexpr int kUmmaK = 32;                          // K of one kind::f8f6f4 instruction
-constexpr int kAStage = kTM * kTK, kBStage = kTN * kTK;
+constexpr int kAStage = kTM * kTK;
 constexpr int kEpiWarps = 8;                        // two per TMEM lane quarter, each taking half of the columns
 constexpr int kTcThreads = 64 + 32 * kEpiWarps;      // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-9: epilogue
 constexpr int kBarrierBytes = 256;
 constexpr int kEpiBufBytes = 32 * 128;              // one staged 32-row x 32-column chunk (FP32; BF16 uses half of it)
 constexpr int kEpiBytes = kEpiWarps * kEpiBufBytes;  // one staging buffer per epilogue warp
 constexpr int kRefBBytes = 2 * kTN * 4;             // refB of the current and the next tile
+// CG = 1: one CTA per 128 x 256 tile, 4 stages of (A 128 x 128 + B 256 x 128) bytes.
+// CG = 2: a pair of CTAs (cta_group::2) per 256 x 256 tile; each CTA stages its 128 rows of A and its 128-row half of
+//         B, 6 stages of 32 KB: a third less shared-memory fill per MMA cycle, which is what bounds the main loop.
+template <int CG> struct TcCfg {
+    static constexpr int kBRows = CG == 2 ? 128 : 256;
+    static constexpr int kBStage = kBRows * kTK;
+    static constexpr int kStages = CG == 2 ? 6 : 4;
+    static constexpr int kRing = kStages * (kAStage + kBStage);
+};
+static_assert(TcCfg<1>::kRing == TcCfg<2>::kRing, "both configurations use the same ring size");
+constexpr int kMaxStages = 6;
 // layout: operand ring | epilogue staging | refB | barriers.  The dynamic shared-memory base is 1024-byte aligned.
-constexpr int kOffEpi = kStages * (kAStage + kBStage);
+constexpr int kOffEpi = TcCfg<1>::kRing;
 constexpr int kOffRefB = kOffEpi + kEpiBytes;
 constexpr int kOffBars = kOffRefB + kRefBBytes;
 constexpr int kTcSmem = kOffBars + kBarrierBytes;
@@ -120,14 +132,71 @@ __global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Completion of all MMAs issued so far by this thread -> one arrival on a barrier of this CTA (CG = 1) or on the barrier
+// at the same offset in both CTAs of the pair (CG = 2: the commit is multicast to the pair; no data moves).
+template <int CG>
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (CG == 1)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
 
+template <int CG>
 __device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    if (CG == 1)
+        asm volatile(
+            "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p; }"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile(
+            "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p; }"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+template <int CG>
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+    if (CG == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+}
+template <int CG>
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    if (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// Address of the same shared-memory location in another CTA of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+// TMA tile load of a CTA pair: data lands in this CTA, the completion is signalled on a barrier of either CTA of the pair.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, uint32_t cluster_bar) {
     asm volatile(
-        "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p; }"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
 }
 
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -154,8 +223,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
     return d;
 }
 
-// kind::f8f6f4, A = B = E5M2, D = F32, both K-major, M = 128, N = 256.
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTN >> 3) << 17) | ((uint32_t)(kTM >> 4) << 24);
+// kind::f8f6f4, A = B = E5M2, D = F32, both K-major, N = 256, M = 128 (one CTA) or 256 (CTA pair).
+template <int CG> struct InstrDesc {
+    static constexpr uint32_t value =
+        (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTN >> 3) << 17) | ((uint32_t)((kTM * CG) >> 4) << 24);
+};
 
 // ------------------------------------------------------------------------------------------------------------------
 // GEMM
@@ -181,12 +253,16 @@ struct TileInfo {
     int kb0, nkb;
 };
 
-__device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile) {
+// Tile `tile` of the launch, as seen by the CTA of rank `rank` in its group of CG CTAs: the group owns a
+// (CG * 128) x 256 output tile, the CTA the 128 rows [m0, m0 + 128) of it and, for CG = 2, the 128-row half
+// [b_half0, b_half0 + 128) of the B tile.
+template <int CG>
+__device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile, int rank) {
     TileInfo t;
     const int per_group = P.mt * P.nt;
     const int g = (P.mode == 2) ? tile / per_group : 0;
     const int rem = tile - g * per_group;
-    t.m0 = (int64_t)(rem / P.nt) * kTM;
+    t.m0 = (int64_t)(rem / P.nt) * (kTM * CG) + (int64_t)rank * kTM;
     t.n0 = (int64_t)(rem % P.nt) * kTN;
     t.b_row0 = 0;
     t.c_row0 = 0;
@@ -207,29 +283,38 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile) {
     return t;
 }
 
+template <int CG>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const TcParams P) {
+    using Cfg = TcCfg<CG>;
+    constexpr int kStages = Cfg::kStages, kBStage = Cfg::kBStage;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t base = smem_u32(smem);
     const uint32_t sA = base, sB = base + kStages * kAStage;
     const uint32_t bars = base + kOffBars;
-    const uint32_t full_bar = bars, empty_bar = bars + 8 * kStages;
-    const uint32_t tfull_bar = bars + 16 * kStages, tempty_bar = tfull_bar + 16;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kOffBars + 16 * kStages + 32);
+    const uint32_t full_bar = bars, empty_bar = bars + 8 * kMaxStages;
+    const uint32_t tfull_bar = bars + 16 * kMaxStages, tempty_bar = tfull_bar + 16;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kOffBars + 16 * kMaxStages + 32);
     volatile uint32_t *abort_flag = tmem_slot + 1;
-    const uint32_t rb_bar = bars + 104;
+    const uint32_t rb_bar = bars + 16 * kMaxStages + 40;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // position in the group of CG CTAs that share an output tile; rank 0 issues the MMAs and owns the barriers the
+    // pair synchronises on (operands landed, accumulator drained)
+    const int rank = CG == 2 ? (int)cluster_cta_rank() : 0;
+    const int group_id = blockIdx.x / CG, num_groups_launched = gridDim.x / CG;
+    const uint32_t lead_full_bar = CG == 2 ? map_to_cta(full_bar, 0) : full_bar;
+    const uint32_t lead_tempty_bar = CG == 2 ? map_to_cta(tempty_bar, 0) : tempty_bar;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(full_bar + 8 * s, CG);            // one arrive.expect_tx per CTA of the group
             mbar_init(empty_bar + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar + 8 * a, 1);
-            mbar_init(tempty_bar + 8 * a, kEpiWarps);
+            mbar_init(tempty_bar + 8 * a, CG * kEpiWarps);
             mbar_init(rb_bar + 8 * a, 32 * kEpiWarps);
         }
         *abort_flag = (base & 1023u) ? 1u : 0u;      // the swizzled layouts below need the 1024-byte alignment
@@ -237,40 +322,48 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     if (warp == 1) {
         __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc<CG>(smem_u32((const void *)tmem_slot), kTmemCols);
     }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();                   // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
         if (lane == 0) {
-            // ---------------- TMA producer
+            // ---------------- TMA producer: this CTA's 128 rows of A and its part of B
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
-                const TileInfo t = tile_info(P, tile);
+            for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+                const TileInfo t = tile_info<CG>(P, tile, rank);
                 for (int kb = 0; kb < t.nkb; ++kb) {
                     if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(full_bar + 8 * stage, kAStage + kBStage);
                     const int32_t kc = (t.kb0 + kb) * kTK;
-                    tma_load_2d(sA + stage * kAStage, &tmA, kc, (int32_t)t.m0, full_bar + 8 * stage);
-                    tma_load_2d(sB + stage * kBStage, &tmB, kc, (int32_t)(t.b_row0 + t.n0), full_bar + 8 * stage);
+                    if (CG == 1) {
+                        mbar_expect_tx(full_bar + 8 * stage, kAStage + kBStage);
+                        tma_load_2d(sA + stage * kAStage, &tmA, kc, (int32_t)t.m0, full_bar + 8 * stage);
+                        tma_load_2d(sB + stage * kBStage, &tmB, kc, (int32_t)(t.b_row0 + t.n0), full_bar + 8 * stage);
+                    } else {
+                        const uint32_t fb = lead_full_bar + 8 * stage;
+                        if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, kAStage + kBStage);
+                        else mbar_expect_tx_cluster(fb, kAStage + kBStage);
+                        tma_load_2d_pair(sA + stage * kAStage, &tmA, kc, (int32_t)t.m0, fb);
+                        tma_load_2d_pair(sB + stage * kBStage, &tmB, kc, (int32_t)(t.b_row0 + t.n0 + rank * Cfg::kBRows), fb);
+                    }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
+        if (lane == 0 && rank == 0) {
+            // ---------------- MMA issuer (rank 0 of the group)
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
-                const TileInfo t = tile_info(P, tile);
+            for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+                const TileInfo t = tile_info<CG>(P, tile, rank);
                 if (t.nkb == 0) continue;
                 if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -283,14 +376,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int k = 0; k < kTK / kUmmaK; ++k) {
                         // advancing K inside the 128-byte swizzle span: +32 bytes = +2 in the (address >> 4) field
-                        tc_mma_f8(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), kInstrDesc,
-                                  (kb > 0 || k > 0) ? 1u : 0u);
+                        tc_mma_f8<CG>(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), InstrDesc<CG>::value,
+                                      (kb > 0 || k > 0) ? 1u : 0u);
                     }
-                    tc_commit(empty_bar + 8 * stage);      // the stage is free once these MMAs have read it
+                    tc_commit<CG>(empty_bar + 8 * stage);  // the stage is free (in every CTA of the group) once read
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit(tfull_bar + 8 * acc);            // accumulator complete
+                tc_commit<CG>(tfull_bar + 8 * acc);        // accumulator complete (in every CTA of the group)
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1u;
             }
@@ -309,8 +402,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int acc = 0, rbuf = 0;
         uint32_t acc_phase = 0, rb_phase[2] = {0u, 0u};
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
-            const TileInfo t = tile_info(P, tile);
+        for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+            const TileInfo t = tile_info<CG>(P, tile, rank);
             const int64_t m_own = t.m0 + q * 32 + lane;
             const float ra = m_own < P.M ? P.refA[m_own] : 0.0f;
             // refB of this tile's 256 columns into shared memory (one value per thread), double-buffered across tiles
@@ -343,7 +436,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // every column of this accumulator has been read: hand it back to the MMA warp
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);
+                        if (lane == 0) {
+                            if (CG == 1) mbar_arrive(tempty_bar + 8 * acc);
+                            else mbar_arrive_cluster(lead_tempty_bar + 8 * acc);
+                        }
                     }
                 } else {
 #pragma unroll
@@ -413,6 +509,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ---------------- teardown
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();                   // neither CTA leaves while the other may still signal its barriers
     if (*abort_flag) {
         // a bounded wait gave up: let any copy still in flight land before shared memory is released
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
@@ -421,7 +518,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        tmem_dealloc<CG>(tmem_base, kTmemCols);
     }
 }
 
@@ -485,8 +582,11 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     decode_rows_kernel<<<(unsigned)decode_ctas, 256, 0, st>>>(D);
     if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
 
+    // CTA pairs (cta_group::2) wherever a 256-row output tile cannot straddle two row groups
+    const int cg = (mode == 1) ? 1 : 2;
     CUtensorMap tmA, tmB;
-    if (!make_map(&tmA, A8, A->rows, K, kTM) || !make_map(&tmB, B8, B->rows, K, kTN)) return UFP4_ERR_CUDA;
+    if (!make_map(&tmA, A8, A->rows, K, kTM) || !make_map(&tmB, B8, B->rows, K, cg == 2 ? TcCfg<2>::kBRows : TcCfg<1>::kBRows))
+        return UFP4_ERR_CUDA;
 
     // C as [groups][rows][cols] so that the TMA store clips at the end of each group's rows and at N
     CUtensorMap tmC;
@@ -510,27 +610,47 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     P.M = M; P.N = N; P.K = K; P.mode = mode;
     P.offsets = offsets; P.num_groups = num_groups; P.group_n = group_n;
     P.refA = refA; P.refB = refB; P.dev_status = dev_status;
-    P.mt = (int)((M + kTM - 1) / kTM);
+    P.mt = (int)((M + kTM * cg - 1) / (kTM * cg));
     P.nt = (int)((N + kTN - 1) / kTN);
     const int64_t total = (int64_t)P.mt * P.nt * (mode == 2 ? num_groups : 1);
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
 
-    static int num_sms = 0;
-    static bool attr_set = false;
+    static int num_sms = 0, max_pairs = 0;
     if (!num_sms) {
         int dev = 0;
         UFP4_CUDA_OK(cudaGetDevice(&dev));
         UFP4_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
+        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
+        // how many CTA pairs can be resident at once (an SM whose neighbour is unavailable cannot host half a pair)
+        cudaLaunchConfig_t probe = {};
+        cudaLaunchAttribute pattr[1];
+        pattr[0].id = cudaLaunchAttributeClusterDimension;
+        pattr[0].val.clusterDim.x = 2; pattr[0].val.clusterDim.y = 1; pattr[0].val.clusterDim.z = 1;
+        probe.gridDim = dim3(2 * (num_sms / 2)); probe.blockDim = dim3(kTcThreads); probe.dynamicSmemBytes = kTcSmem;
+        probe.attrs = pattr; probe.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&max_pairs, gemm_tc_kernel<2>, &probe) != cudaSuccess || max_pairs < 1)
+            max_pairs = num_sms / 2;
+        if (getenv("UFP4_DEBUG")) fprintf(stderr, "[ufp4] SMs %d, resident CTA pairs %d\n", num_sms, max_pairs);
     }
-    if (!attr_set) {
-        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
-        attr_set = true;
+    if (cg == 1) {
+        const int grid = (int)(total < num_sms ? total : num_sms);
+        gemm_tc_kernel<1><<<grid, kTcThreads, kTcSmem, st>>>(tmA, tmB, tmC, P);
+        return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
     }
-    const int grid = (int)(total < num_sms ? total : num_sms);
-    gemm_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(tmA, tmB, tmC, P);
-    return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(2 * (unsigned)(total < max_pairs ? total : max_pairs));
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kTcSmem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, tmA, tmB, tmC, P) == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------------------------
