@@ -6,10 +6,11 @@
 // in E5M2 once a per-row reference exponent is factored out.  Two kernels:
 //   1. decode_rows_kernel: packed nibbles + scales  ->  E5M2 bytes [rows][K] and one FP32 reference scale per row
 //      (caller's workspace); blocks more than 2^26 below the row's largest block are flushed and reported.
-//   2. gemm_tc_kernel: persistent, warp-specialised.  One thread issues TMA tile loads (128B-swizzled, 4-stage ring),
-//      one thread issues tcgen05.mma kind::f8f6f4 (M128 x N256 x K32) into a double-buffered FP32 accumulator in
-//      tensor memory, four warps drain accumulators with tcgen05.ld, apply refA[m] * refB[n] and store C.
-// Every products q_a 2^ea * q_b 2^eb is exact; accumulation is the tensor core's FP32.
+//   2. gemm_tc_kernel: persistent, warp-specialised.  One thread issues TMA tile loads (128B-swizzled ring), one thread
+//      issues tcgen05.mma kind::f8f6f4 (N256 x K32; M128 per CTA, or M256 on a CTA pair with cta_group::2) into a
+//      double-buffered FP32 accumulator in tensor memory, eight warps drain accumulators with tcgen05.ld, apply
+//      refA[m] * refB[n] and hand 32 x 32 boxes of C to TMA stores.
+// Every product q_a 2^ea * q_b 2^eb is exact; accumulation is the tensor core's FP32.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdio.h>
@@ -97,13 +98,16 @@ __global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) 
     const uint32_t lut_lo0 = 0x42403C00u;                                           // entries 3, 2, 1, 0
     const uint32_t lut_hi0 = O.grid == UFP4_GRID_E2M1 ? 0x4A484644u : 0x47464544u;  // entries 7, 6, 5, 4
     bool flushed = false;
-    const uint8_t *crow = O.codes + row * O.ldc;
-    uint8_t *orow = O.out8 + row * P.K;
-    for (int64_t kb = lane; kb < nkb; kb += 32) {
-        const uint32_t sb = __float_as_uint(srow[kb]);
-        const uint2 cw = *reinterpret_cast<const uint2 *>(crow + kb * 8);
+    const int nkb32 = (int)nkb;
+    const uint2 *cptr = reinterpret_cast<const uint2 *>(O.codes + row * O.ldc) + lane;
+    uint4 *optr = reinterpret_cast<uint4 *>(O.out8 + row * P.K) + lane;
+    const float *sptr = srow + lane;
+#pragma unroll 4
+    for (int kb = lane; kb < nkb32; kb += 32, cptr += 32, optr += 32, sptr += 32) {
+        const uint32_t sb = __float_as_uint(__ldg(sptr));
+        const uint2 cw = __ldg(cptr);
         uint32_t out[4] = {0u, 0u, 0u, 0u};
-        const int d = (int)((sb >> 23) & 0xFFu) - 127 - eref;
+        const int d = (int)(sb >> 23) - 127 - eref;       // scales are non-negative: no sign bit to mask
         if (sb != 0u && d < kDMin) {
             flushed |= (cw.x | cw.y) != 0u;
         } else if (sb != 0u) {
@@ -118,13 +122,12 @@ __global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) 
                     const uint32_t m = (w & 0x88888888u) >> 3;
                     w = (w ^ (m * 7u)) + m;
                 }
-                const uint32_t mag_lo = w & 0x7777u, mag_hi = (w >> 16) & 0x7777u;
-                const uint32_t sg_lo = (w >> 3) & 0x1111u, sg_hi = (w >> 19) & 0x1111u;
-                out[2 * h] = __byte_perm(lut_lo, lut_hi, mag_lo) | __byte_perm(0x00008000u, 0u, sg_lo);
-                out[2 * h + 1] = __byte_perm(lut_lo, lut_hi, mag_hi) | __byte_perm(0x00008000u, 0u, sg_hi);
+                // byte k of the result: table[magnitude of nibble k] | sign of nibble k << 7 (both by byte permutes)
+                out[2 * h] = __byte_perm(lut_lo, lut_hi, w & 0x7777u) | __byte_perm(0x00008000u, 0u, (w >> 3) & 0x1111u);
+                out[2 * h + 1] = __byte_perm(lut_lo, lut_hi, (w >> 16) & 0x7777u) | __byte_perm(0x00008000u, 0u, (w >> 19) & 0x1111u);
             }
         }
-        *reinterpret_cast<uint4 *>(orow + kb * 16) = make_uint4(out[0], out[1], out[2], out[3]);
+        *optr = make_uint4(out[0], out[1], out[2], out[3]);
     }
     if (flushed && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
 }
