@@ -70,7 +70,8 @@ class Ufp4MoE:
 
     def __init__(self, offsets_host: torch.Tensor, hidden: int, ffn: int, device="cuda", grid: int = ufp4.GRID_INT4,
                  scale_fmt: int = ufp4.SCALE_FP32, path: int = ufp4.PATH_AUTO, rht_block: int = 16, seed_rht: int = 1,
-                 seed_sr: int = 2, out_bf16: bool = False):
+                 seed_sr: int = 2, out_bf16: bool = False, counts: torch.Tensor | None = None):
+        self.counts = counts
         self.offsets_host = offsets_host.to(torch.int64).contiguous()
         self.offsets_dev = self.offsets_host.to(device)
         E, R, H, F = offsets_host.numel() - 1, int(offsets_host[-1]), hidden, ffn
@@ -109,6 +110,12 @@ class Ufp4MoE:
         self.gemms(stream)
         return self.Y, self.dX, self.dW
 
-    def flops(self, counts: torch.Tensor) -> int:
-        """Useful flops: unpadded routed rows only."""
-        return 3 * 2 * int(counts.sum()) * self.H * self.F
+    @property
+    def flops(self) -> int:
+        """Useful flops: unpadded routed rows only (padded rows if the counts were not given)."""
+        rows = int(self.counts.sum()) if self.counts is not None else self.R
+        return 3 * 2 * rows * self.H * self.F
+
+    @property
+    def quantize_elements(self) -> int:
+        return self.R * self.H + self.E * self.F * self.H + self.R * self.F
