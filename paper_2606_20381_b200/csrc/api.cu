@@ -17,6 +17,12 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
                        int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                        void *stream);
 
+size_t gemm_promote_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
+int gemm_promote_kernel_launches();
+int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
+                        int64_t M, int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n,
+                        void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
 static int check_operand(const ufp4_qtensor *q) {
     if (!q || !q->codes || !q->scales) return UFP4_ERR_NULL;
     if (q->grid < 0 || q->grid > 2 || q->scale_fmt < 0 || q->scale_fmt > 2) return UFP4_ERR_ENUM;
@@ -32,21 +38,30 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                          int mode, int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                          int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                          void *stream) {
-    if (path < 0 || path > 2) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 3) return UFP4_ERR_ENUM;
     if (!C) return UFP4_ERR_NULL;
     if (ldc < N) return UFP4_ERR_SHAPE;
     if (!aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
-    bool tensor_ok = gemm_tensor_supported(A, B, M, N, K, mode);
+    const bool tensor_ok = gemm_tensor_supported(A, B, M, N, K, mode);
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
-    if (path == UFP4_PATH_EXACT || !tensor_ok)
+    if (path == UFP4_PATH_EXACT)
         return gemm_exact_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, stream);
-    size_t need = gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
-    if (!workspace || workspace_bytes < need) {
+    if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) {
+        const size_t need = gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
+        if (workspace && workspace_bytes >= need)
+            return gemm_tensor_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
+                                      workspace, workspace_bytes, dev_status, stream);
         if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
-        return gemm_exact_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, stream);
     }
-    return gemm_tensor_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
-                              workspace, workspace_bytes, dev_status, stream);
+    // PROMOTE, or AUTO for scale formats the folded path cannot take
+    {
+        const size_t need = gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
+        if (workspace && workspace_bytes >= need)
+            return gemm_promote_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, workspace,
+                                       workspace_bytes, dev_status, stream);
+        if (path == UFP4_PATH_PROMOTE) return UFP4_ERR_WORKSPACE;
+    }
+    return gemm_exact_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, stream);
 }
 
 }  // namespace ufp4
@@ -79,8 +94,10 @@ extern "C" int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t
 
 extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path) {
     if (!A || !B || path == UFP4_PATH_EXACT) return 0;
-    if (A->scale_fmt != UFP4_SCALE_POW2 || B->scale_fmt != UFP4_SCALE_POW2) return 0;
-    return ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
+    const bool pow2 = A->scale_fmt == UFP4_SCALE_POW2 && B->scale_fmt == UFP4_SCALE_POW2;
+    if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
+        return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
+    return ufp4::gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
 }
 
 extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B, int path, int *kernel_launches) {
@@ -88,12 +105,15 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (rc != UFP4_OK) return rc;
     rc = ufp4::check_operand(B);
     if (rc != UFP4_OK) return rc;
-    if (path < 0 || path > 2) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 3) return UFP4_ERR_ENUM;
     if (A->k != B->k) return UFP4_ERR_SHAPE;
     bool tensor_ok = ufp4::gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0);
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
-    int taken = (path == UFP4_PATH_EXACT || !tensor_ok) ? UFP4_PATH_EXACT : UFP4_PATH_TENSOR;
-    if (kernel_launches) *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : ufp4::gemm_tensor_kernel_launches();
+    int taken = path == UFP4_PATH_EXACT ? UFP4_PATH_EXACT
+              : (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) ? UFP4_PATH_TENSOR : UFP4_PATH_PROMOTE;
+    if (kernel_launches)
+        *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : taken == UFP4_PATH_TENSOR ? ufp4::gemm_tensor_kernel_launches()
+                                                                                     : ufp4::gemm_promote_kernel_launches();
     return taken;
 }
 

@@ -18,10 +18,10 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "tc.cuh"
 
 namespace ufp4 {
 
-constexpr int kTM = 128, kTN = 256, kTK = 128;     // per-CTA output tile (bytes along K: one E5M2 byte per element)
 constexpr int kUmmaK = 32;                          // K of one kind::f8f6f4 instruction
 constexpr int kAStage = kTM * kTK;
 constexpr int kEpiWarps = 8;                        // two per TMEM lane quarter, each taking half of the columns
@@ -130,160 +130,6 @@ __global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) 
         *optr = make_uint4(out[0], out[1], out[2], out[3]);
     }
     if (flushed && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Completion of all MMAs issued so far by this thread -> one arrival on a barrier of this CTA (CG = 1) or on the barrier
-// at the same offset in both CTAs of the pair (CG = 2: the commit is multicast to the pair; no data moves).
-template <int CG>
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    if (CG == 1)
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-    else
-        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                     ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-
-template <int CG>
-__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    if (CG == 1)
-        asm volatile(
-            "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p; }"
-            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-    else
-        asm volatile(
-            "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p; }"
-            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-template <int CG>
-__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
-    if (CG == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    } else {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
-}
-template <int CG>
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    if (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-
-// Address of the same shared-memory location in another CTA of the cluster.
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
-}
-// TMA tile load of a CTA pair: data lands in this CTA, the completion is signalled on a barrier of either CTA of the pair.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, uint32_t cluster_bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(cluster_bar) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t cluster_cta_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// K-major, 128B-swizzled shared-memory operand: rows of 128 bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);          // start address
-    d |= (uint64_t)1u << 16;                          // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024u >> 4) << 32;                // stride byte offset between 8-row groups
-    d |= (uint64_t)1u << 46;                          // descriptor version of this architecture
-    d |= (uint64_t)2u << 61;                          // 128-byte swizzle
-    return d;
-}
-
-// kind::f8f6f4, A = B = E5M2, D = F32, both K-major, N = 256, M = 128 (one CTA) or 256 (CTA pair).
-template <int CG> struct InstrDesc {
-    static constexpr uint32_t value =
-        (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTN >> 3) << 17) | ((uint32_t)((kTM * CG) >> 4) << 24);
-};
-
-// ------------------------------------------------------------------------------------------------------------------
-// GEMM
-// ------------------------------------------------------------------------------------------------------------------
-
-struct TcParams {
-    void *C;
-    int64_t ldc;
-    int c_is_bf16;
-    int64_t M, N, K;          // tile space M x N; K is the whole reduction length of the operands
-    int mode;                 // 0 plain, 1 rows grouped, 2 reduction grouped
-    const int64_t *offsets;
-    int num_groups;
-    int64_t group_n;
-    const float *refA, *refB;
-    int32_t *dev_status;
-    int mt, nt, total_tiles;
-    int n_unaligned;          // N * sizeof(element of C) is not a multiple of 16
-};
-
-struct TileInfo {
-    int64_t m0, n0, b_row0, c_row0;
-    int kb0, nkb;
-};
-
-// Tile `tile` of the launch, as seen by the CTA of rank `rank` in its group of CG CTAs: the group owns a
-// (CG * 128) x 256 output tile, the CTA the 128 rows [m0, m0 + 128) of it and, for CG = 2, the 128-row half
-// [b_half0, b_half0 + 128) of the B tile.
-template <int CG>
-__device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile, int rank) {
-    TileInfo t;
-    const int per_group = P.mt * P.nt;
-    const int g = (P.mode == 2) ? tile / per_group : 0;
-    const int rem = tile - g * per_group;
-    t.m0 = (int64_t)(rem / P.nt) * (kTM * CG) + (int64_t)rank * kTM;
-    t.n0 = (int64_t)(rem % P.nt) * kTN;
-    t.b_row0 = 0;
-    t.c_row0 = 0;
-    t.kb0 = 0;
-    t.nkb = (int)((P.K + kTK - 1) / kTK);
-    if (P.mode == 1) {
-        int lo = 0, hi = P.num_groups;
-        while (hi - lo > 1) {
-            int mid = (lo + hi) >> 1;
-            if (P.offsets[mid] <= t.m0) lo = mid; else hi = mid;
-        }
-        t.b_row0 = (int64_t)lo * P.group_n;
-    } else if (P.mode == 2) {
-        t.kb0 = (int)(P.offsets[g] / kTK);
-        t.nkb = (int)((P.offsets[g + 1] - P.offsets[g]) / kTK);
-        t.c_row0 = (int64_t)g * P.M;
-    }
-    return t;
 }
 
 template <int CG>

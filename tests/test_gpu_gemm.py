@@ -22,7 +22,7 @@ def three_products(X, W, dY, grid, scale_fmt=oracle.SCALE_FP32, seed_rht=1, seed
     return {"fwd_y": (Xr, Wr, ufp4.FWD_Y), "bwd_dx": (Gr, Wc, ufp4.BWD_DX), "bwd_dw": (Gc, Xc, ufp4.BWD_DW)}
 
 
-@pytest.mark.parametrize("path", [ufp4.PATH_EXACT])
+@pytest.mark.parametrize("path", [ufp4.PATH_EXACT, ufp4.PATH_PROMOTE])
 @pytest.mark.parametrize("grid", [oracle.GRID_INT4, oracle.GRID_E1M2, oracle.GRID_E2M1])
 def test_tiny_layer_all_three_products(grid, path):
     X, W, dY = inputs.tiny_layer(0)
@@ -38,8 +38,9 @@ def test_tiny_layer_all_three_products(grid, path):
     assert np.linalg.norm(got - exact) / np.linalg.norm(exact) < 0.2
 
 
+@pytest.mark.parametrize("path", [ufp4.PATH_EXACT, ufp4.PATH_PROMOTE])
 @pytest.mark.parametrize("scale_fmt", [oracle.SCALE_FP32, oracle.SCALE_POW2, oracle.SCALE_E4M3_TENSOR])
-def test_ragged_shapes_and_scale_formats_exact_path(scale_fmt):
+def test_ragged_shapes_and_scale_formats_exact_path(scale_fmt, path):
     M, N, K = 200, 72, 176
     X = inputs.heavy_tailed_activations(M, K, seed=21)
     W = inputs.normal_bf16(N, K, 0.02, seed=22)
@@ -51,12 +52,35 @@ def test_ragged_shapes_and_scale_formats_exact_path(scale_fmt):
     A = oracle_quantize(X, oracle.AXIS_ROW, grid=oracle.GRID_INT4, **kwx)
     B = oracle_quantize(W, oracle.AXIS_ROW, grid=oracle.GRID_E2M1, **kww)        # mixed grids are allowed
     ref, S = oracle.gemm(A, B)
-    got = ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_EXACT).cpu().numpy()
+    got = ufp4.gemm(to_device(A), to_device(B), path=path).cpu().numpy()
     assert_gemm_close(got, ref, S, f"ragged fmt {scale_fmt}")
     out = torch.full((M, 80), 7.0, dtype=torch.bfloat16, device="cuda")        # BF16 output into a padded buffer
-    ufp4.gemm(to_device(A), to_device(B), out=out[:, :N], path=ufp4.PATH_EXACT)
+    ufp4.gemm(to_device(A), to_device(B), out=out[:, :N], path=path)
     assert_gemm_close(out[:, :N].float().cpu().numpy(), ref, S, "bf16 out", bf16_out=True)
     assert torch.all(out[:, N:] == 7.0)
+
+
+@pytest.mark.parametrize("shape", [(130, 260, 144), (384, 512, 1040), (1, 1, 16), (128, 128, 4096), (1024, 1536, 2048)])
+def test_promote_path_shapes(shape):
+    """The tensor-core + promotion path for FP32 scales over ragged, multi-tile and long-K shapes."""
+    M, N, K = shape
+    X = inputs.heavy_tailed_activations(M, K, seed=21)
+    W = inputs.normal_bf16(N, K, 0.02, seed=22)
+    A = oracle_quantize(X, oracle.AXIS_ROW, rht_block=16, scale_fmt=oracle.SCALE_FP32, seed_rht=5)
+    B = oracle_quantize(W, oracle.AXIS_ROW, rht_block=16, scale_fmt=oracle.SCALE_FP32, seed_rht=5)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_PROMOTE, dev_status=status)
+    assert int(status.item()) == 0
+    if M * N <= 1 << 19:
+        ref, S = oracle.gemm(A, B)
+        assert_gemm_close(out.cpu().numpy(), ref, S, f"promote {shape}")
+    else:
+        rng = np.random.default_rng(7)
+        im, in_ = rng.integers(0, M, 20000), rng.integers(0, N, 20000)
+        c, s = oracle.gemm_sampled(A, B, im, in_)
+        assert_gemm_close(out.cpu().numpy()[im, in_], c, s, f"promote sampled {shape}")
+    assert torch.equal(out, ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_PROMOTE))
+    assert ufp4.gemm_path_name(to_device(A), to_device(B), ufp4.PATH_AUTO) == "promote"
 
 
 def test_integer_and_one_hot_operands():
@@ -112,9 +136,10 @@ def test_grouped_products_small():
     cases = {"fwd_y": (Xr, Wr, ufp4.FWD_Y, F), "bwd_dx": (Gr, Wc, ufp4.BWD_DX, H), "bwd_dw": (Gc, Xc, ufp4.BWD_DW, F)}
     for name, (A, B, layout, gn) in cases.items():
         ref, S = grouped_reference(A, B, offsets, gn, layout)
-        got = ufp4.gemm_grouped(to_device(A), to_device(B), off_d, off_h, gn, layout, path=ufp4.PATH_EXACT).cpu().numpy()
-        assert got.shape == ref.shape, name
-        assert_gemm_close(got, ref, S, f"grouped {name}")
+        for path in (ufp4.PATH_EXACT, ufp4.PATH_PROMOTE):
+            got = ufp4.gemm_grouped(to_device(A), to_device(B), off_d, off_h, gn, layout, path=path).cpu().numpy()
+            assert got.shape == ref.shape, name
+            assert_gemm_close(got, ref, S, f"grouped {name} path {path}")
     # the empty group's dW is exactly zero
     got = ufp4.gemm_grouped(to_device(Gc), to_device(Xc), off_d, off_h, F, ufp4.BWD_DW, path=ufp4.PATH_EXACT)
     assert torch.all(got[F:2 * F] == 0)
