@@ -69,67 +69,97 @@ struct DecodeParams {
     int32_t *dev_status;
 };
 
-constexpr int kDecodeRowsPerCta = 8;   // one warp per row
+constexpr int kDecodeThreads = 256;
 
-__global__ void __launch_bounds__(256) decode_rows_kernel(const DecodeParams P) {
+// A CTA decodes 256 / TPR rows with TPR threads (32..256) on each: short rows keep a warp per row, long rows are
+// spread over more threads so that the grid has many more warps than the GPU has slots (no idle tail).
+template <int TPR>
+__global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const DecodeParams P) {
+    __shared__ int s_emax[kDecodeThreads / 32];
+    constexpr int kRowsPerCta = kDecodeThreads / TPR, kWarpsPerRow = TPR / 32;
     const bool is_b = (int64_t)blockIdx.x >= P.a_ctas;
     const DecodeOperand &O = P.op[is_b ? 1 : 0];
-    const int lane = threadIdx.x & 31;
-    const int64_t row = ((int64_t)blockIdx.x - (is_b ? P.a_ctas : 0)) * kDecodeRowsPerCta + (threadIdx.x >> 5);
-    if (row >= O.rows) return;
-    const int64_t nkb = P.K >> 4;
-    const float *srow = O.scales + row * O.lds;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = threadIdx.x % TPR;
+    const int64_t row = ((int64_t)blockIdx.x - (is_b ? P.a_ctas : 0)) * kRowsPerCta + threadIdx.x / TPR;
+    const bool active = row < O.rows;
+    const int nkb = (int)(P.K >> 4);
+    const float *sptr = O.scales + (active ? row : 0) * O.lds + t;
 
-    // largest block exponent of the row (power-of-two scales: the exponent field is the scale)
-    int emax = -1000;
-    for (int64_t kb = lane; kb < nkb; kb += 32) {
-        const uint32_t b = __float_as_uint(srow[kb]);
-        if (b != 0u) emax = max(emax, (int)((b >> 23) & 0xFFu) - 127);
+    // largest block exponent field of the row (power-of-two scales: the exponent field is the scale; 0 = zero block)
+    uint32_t fmax = 0u;
+    if (active) {
+        // eight loads in flight per thread: the row's scales are the first touch of DRAM, and a warp issues in order
+        int kb = t;
+        for (; kb + 7 * TPR < nkb; kb += 8 * TPR) {
+            uint32_t b[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) b[u] = __float_as_uint(__ldg(sptr + (kb - t) + u * TPR));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) fmax = max(fmax, b[u]);
+        }
+        for (; kb < nkb; kb += TPR) fmax = max(fmax, __float_as_uint(__ldg(sptr + (kb - t))));
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, o));
-    if (emax == -1000) emax = kDMax;                 // all-zero row
-    const int eref = emax - kDMax;
-    const float unit = O.grid == UFP4_GRID_INT4 ? 1.0f : (O.grid == UFP4_GRID_E1M2 ? 0.25f : 0.5f);
-    if (lane == 0) O.ref[row] = ldexpf(unit, eref);
-
-    // E5M2 bytes of the magnitudes 1..7 of a grid at d = 0, i.e. mag = 2^k (1 + f/4) -> (15 + k) << 2 | f; entry 0 is 0.
-    // Uniform grids: 1, 2, 3, 4, 5, 6, 7.  E2M1 (2 * value): 1, 2, 3, 4, 6, 8, 12.
-    const uint32_t lut_lo0 = 0x42403C00u;                                           // entries 3, 2, 1, 0
-    const uint32_t lut_hi0 = O.grid == UFP4_GRID_E2M1 ? 0x4A484644u : 0x47464544u;  // entries 7, 6, 5, 4
-    bool flushed = false;
-    const int nkb32 = (int)nkb;
-    const uint2 *cptr = reinterpret_cast<const uint2 *>(O.codes + row * O.ldc) + lane;
-    uint4 *optr = reinterpret_cast<uint4 *>(O.out8 + row * P.K) + lane;
-    const float *sptr = srow + lane;
-#pragma unroll 4
-    for (int kb = lane; kb < nkb32; kb += 32, cptr += 32, optr += 32, sptr += 32) {
-        const uint32_t sb = __float_as_uint(__ldg(sptr));
-        const uint2 cw = __ldg(cptr);
-        uint32_t out[4] = {0u, 0u, 0u, 0u};
-        const int d = (int)(sb >> 23) - 127 - eref;       // scales are non-negative: no sign bit to mask
-        if (sb != 0u && d < kDMin) {
-            flushed |= (cw.x | cw.y) != 0u;
-        } else if (sb != 0u) {
-            // per-block lookup table: 4 d is added to each non-zero entry; every byte stays inside [4, 0x7A], so the
-            // 32-bit wrap-around arithmetic below is an exact per-byte addition also for negative d
-            const uint32_t off = (uint32_t)(d * 4);
-            const uint32_t lut_lo = lut_lo0 + off * 0x01010100u, lut_hi = lut_hi0 + off * 0x01010101u;
+    for (int o = 16; o > 0; o >>= 1) fmax = max(fmax, __shfl_xor_sync(0xFFFFFFFFu, fmax, o));
+    if (kWarpsPerRow > 1) {
+        if (lane == 0) s_emax[warp] = (int)fmax;
+        __syncthreads();
+        const int w0 = warp / kWarpsPerRow * kWarpsPerRow;      // first warp of this row
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t w = h ? cw.y : cw.x;
-                if (O.grid == UFP4_GRID_INT4) {             // two's complement -> sign | magnitude nibbles
-                    const uint32_t m = (w & 0x88888888u) >> 3;
-                    w = (w ^ (m * 7u)) + m;
-                }
-                // byte k of the result: table[magnitude of nibble k] | sign of nibble k << 7 (both by byte permutes)
-                out[2 * h] = __byte_perm(lut_lo, lut_hi, w & 0x7777u) | __byte_perm(0x00008000u, 0u, (w >> 3) & 0x1111u);
-                out[2 * h + 1] = __byte_perm(lut_lo, lut_hi, (w >> 16) & 0x7777u) | __byte_perm(0x00008000u, 0u, (w >> 19) & 0x1111u);
-            }
+        for (int w = 0; w < kWarpsPerRow; ++w) fmax = max(fmax, (uint32_t)s_emax[w0 + w]);
+    }
+    if (!active) return;
+    // biased exponent field of the row's reference 2^eref, eref = emax - kDMax (an all-zero row takes eref = 0)
+    const int fref = fmax == 0u ? 127 : (int)(fmax >> 23) - kDMax;
+    if (t == 0) {
+        // unit * 2^eref as two exact factors (fref may be below the smallest normal exponent field)
+        const float unit = O.grid == UFP4_GRID_INT4 ? 1.0f : (O.grid == UFP4_GRID_E1M2 ? 0.25f : 0.5f);
+        const int h = fref >= 1 ? fref : 1;
+        O.ref[row] = __fmul_rn(__fmul_rn(unit, __uint_as_float((uint32_t)(127 + fref - h) << 23)), __uint_as_float((uint32_t)h << 23));
+    }
+
+    // E5M2 bytes of a grid's values at d = 0: magnitude 2^k (1 + f/4) -> (15 + k) << 2 | f, bit 7 = sign.  A nibble n
+    // indexes a 16-entry table held in four registers: entries 0..7 (n < 8) and 8..15 (n >= 8, index n & 7).
+    // Uniform grids: magnitudes 0..7 (INT4 two's complement: n >= 8 is n - 16, i.e. -8..-1; E1M2: sign | magnitude).
+    // E2M1 (2 * value): 0, 1, 2, 3, 4, 6, 8, 12.  The negative zero of the sign | magnitude grids decodes to 0.
+    const bool int4 = O.grid == UFP4_GRID_INT4;
+    const uint32_t lutp_lo0 = 0x42403C00u;
+    const uint32_t lutp_hi0 = O.grid == UFP4_GRID_E2M1 ? 0x4A484644u : 0x47464544u;
+    const uint32_t lutn_lo0 = int4 ? 0xC5C6C7C8u : (lutp_lo0 | 0x80808000u);
+    const uint32_t lutn_hi0 = int4 ? 0xBCC0C2C4u : (lutp_hi0 | 0x80808080u);
+    const uint32_t mul_nlo = int4 ? 0x04040404u : 0x04040400u;     // a zero entry stays zero
+    const int fkeep = max(1, fref + kDMin);                        // smallest exponent field that is not flushed
+    uint32_t flushed = 0u;
+    const uint2 *cptr = reinterpret_cast<const uint2 *>(O.codes + row * O.ldc) + t;
+    uint4 *optr = reinterpret_cast<uint4 *>(O.out8 + row * P.K) + t;
+#pragma unroll 4
+    for (int kb = t; kb < nkb; kb += TPR, cptr += TPR, optr += TPR, sptr += TPR) {
+        const int f = (int)(__float_as_uint(__ldg(sptr)) >> 23);   // scales are non-negative: no sign bit to mask
+        uint2 cw = __ldg(cptr);
+        // a zero-scale or flushed block decodes as all-zero codes (table entry 0 is 0 at every d)
+        const bool keep = f >= fkeep;
+        flushed |= (keep || f == 0) ? 0u : (cw.x | cw.y);
+        cw.x = keep ? cw.x : 0u;
+        cw.y = keep ? cw.y : 0u;
+        // per-block table: 4 d is added to each non-zero entry; the low 7 bits of every entry stay inside [4, 0x7A], so
+        // the 32-bit wrap-around arithmetic below is an exact per-byte addition also for negative d
+        const uint32_t d = (uint32_t)(f - fref);
+        const uint32_t lutp_lo = lutp_lo0 + d * 0x04040400u, lutp_hi = lutp_hi0 + d * 0x04040404u;
+        const uint32_t lutn_lo = lutn_lo0 + d * mul_nlo, lutn_hi = lutn_hi0 + d * 0x04040404u;
+        uint32_t out[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            // four nibbles: look the low three bits up in both halves of the table, then take byte k from the half that
+            // bit 3 of nibble k names (selector nibble k = k, or 4 + k)
+            const uint32_t w = (q & 2 ? cw.y : cw.x) >> (q & 1 ? 16 : 0);
+            const uint32_t sel = w & 0x7777u;
+            const uint32_t pos = __byte_perm(lutp_lo, lutp_hi, sel), neg = __byte_perm(lutn_lo, lutn_hi, sel);
+            out[q] = __byte_perm(pos, neg, ((w >> 1) & 0x4444u) | 0x3210u);
         }
         *optr = make_uint4(out[0], out[1], out[2], out[3]);
     }
-    if (flushed && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
+    if (flushed != 0u && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
 }
 
 template <int CG>
@@ -424,11 +454,18 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     D.op[1] = DecodeOperand{static_cast<const uint8_t *>(B->codes), static_cast<const float *>(B->scales),
                             B->ld_codes_bytes, B->ld_scales, B->rows, B->grid, B8, refB};
     D.K = K;
-    D.a_ctas = (A->rows + kDecodeRowsPerCta - 1) / kDecodeRowsPerCta;
+    int tpr = 32;           // a warp per row up to 8 blocks per thread, more threads on longer rows
+    while (tpr < kDecodeThreads && (K >> 4) >= (int64_t)16 * tpr) tpr *= 2;
+    const int64_t rows_per_cta = kDecodeThreads / tpr;
+    D.a_ctas = (A->rows + rows_per_cta - 1) / rows_per_cta;
     D.dev_status = dev_status;
-    const int64_t decode_ctas = D.a_ctas + (B->rows + kDecodeRowsPerCta - 1) / kDecodeRowsPerCta;
+    const int64_t decode_ctas = D.a_ctas + (B->rows + rows_per_cta - 1) / rows_per_cta;
     if (decode_ctas > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
-    decode_rows_kernel<<<(unsigned)decode_ctas, 256, 0, st>>>(D);
+    const unsigned dg = (unsigned)decode_ctas;
+    if (tpr == 32) decode_rows_kernel<32><<<dg, kDecodeThreads, 0, st>>>(D);
+    else if (tpr == 64) decode_rows_kernel<64><<<dg, kDecodeThreads, 0, st>>>(D);
+    else if (tpr == 128) decode_rows_kernel<128><<<dg, kDecodeThreads, 0, st>>>(D);
+    else decode_rows_kernel<256><<<dg, kDecodeThreads, 0, st>>>(D);
     if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
 
     // CTA pairs (cta_group::2) wherever a 256-row output tile cannot straddle two row groups

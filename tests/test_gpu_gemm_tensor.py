@@ -127,3 +127,28 @@ def test_grouped_products_small():
         assert_gemm_close(got, ref, S, f"grouped {name}")
     got = ufp4.gemm_grouped(to_device(Gc), to_device(Xc), off_d, off_h, F, ufp4.BWD_DW, path=ufp4.PATH_TENSOR)
     assert torch.all(got[F:2 * F] == 0)
+
+
+@pytest.mark.parametrize("grid", [oracle.GRID_INT4, oracle.GRID_E1M2, oracle.GRID_E2M1])
+@pytest.mark.parametrize("path", [ufp4.PATH_TENSOR, ufp4.PATH_PROMOTE, ufp4.PATH_EXACT])
+def test_every_nibble_code_on_every_path(grid, path):
+    """Hand-made operands holding all 16 nibble codes (also the ones the quantizer never emits: INT4 0x8 = -8, the
+    negative zero of the sign | magnitude grids) with scales spread over the exponent window, zero scales included."""
+    rng = np.random.default_rng(7)
+    M, N, K = 96, 80, 256
+
+    def operand(rows):
+        codes = rng.integers(0, 256, size=(rows, K // 2), dtype=np.uint8)
+        codes[0, :8] = np.arange(8, dtype=np.uint8) * 0x22          # every code twice in row 0: 0x00, 0x22, ..., 0xEE
+        codes[0, 8:16] = np.arange(8, 16, dtype=np.uint8) * 0x11
+        scales = np.ldexp(1.0, rng.integers(-10, 11, size=(rows, K // 16))).astype(np.float32)
+        scales[rng.random(scales.shape) < 0.1] = 0.0
+        return oracle.QTensor(codes, scales, grid, oracle.SCALE_POW2)
+
+    A, B = operand(M), operand(N)
+    c_ref, s_ref = oracle.gemm(A, B)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = ufp4.gemm(to_device(A), to_device(B), path=path, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert_gemm_close(out.cpu().numpy(), c_ref, s_ref, f"grid {grid} path {path}")
