@@ -17,7 +17,7 @@ class Ufp4Linear:
 
     def __init__(self, tokens: int, in_features: int, out_features: int, device="cuda", grid: int = ufp4.GRID_INT4,
                  scale_fmt: int = ufp4.SCALE_FP32, path: int = ufp4.PATH_AUTO, rht_block: int = 16,
-                 seed_rht: int = 1, seed_sr: int = 2, out_bf16: bool = False):
+                 seed_rht: int = 1, seed_sr: int = 2, out_bf16: bool = False, overlap: bool = False):
         T, K, N = tokens, in_features, out_features
         self.T, self.K, self.N = T, K, N
         self.grid, self.scale_fmt, self.path, self.rht_block = grid, scale_fmt, path, rht_block
@@ -34,6 +34,13 @@ class Ufp4Linear:
                    ufp4.gemm_workspace_bytes(self.Gc, self.Xc, path))
         self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
         self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+        # overlap: the three products run on three streams (each with its own workspace), so that the operand
+        # preparation of one product and the tails of the quantizer launches fill SMs another kernel leaves idle
+        self.overlap = overlap
+        if overlap:
+            self.workspaces = [self.workspace] + [torch.empty_like(self.workspace) for _ in range(2)]
+            self.side = [torch.cuda.Stream(device=device) for _ in range(2)]
+            self.ev = {k: torch.cuda.Event() for k in ("start", "x", "w", "g", "dx", "dw")}
 
     # number of kernel launches one call makes (for the benchmark's launch count)
     launches_quantize = 3
@@ -51,10 +58,49 @@ class Ufp4Linear:
         ufp4.gemm(self.Gr, self.Wc, out=self.dX, layout=ufp4.BWD_DX, **kw)
         ufp4.gemm(self.Gc, self.Xc, out=self.dW, layout=ufp4.BWD_DW, **kw)
 
-    def step(self, X, W, dY, stream=None):
+    def step(self, X, W, dY, stream=None, join: bool = True):
+        if self.overlap:
+            return self.step_overlapped(X, W, dY, stream, join)
         self.quantize(X, W, dY, stream)
         self.gemms(stream)
         return self.Y, self.dX, self.dW
+
+    def step_overlapped(self, X, W, dY, stream=None, join: bool = True):
+        """The same six calls as step(), ordered only by their data dependences: X, W and fwd_y on the caller's stream,
+        dY and bwd_dx on a second, bwd_dw on a third; the caller's stream joins both at the end (join=False leaves
+        that to a later join() call, so that independent layers overlap too)."""
+        s0 = torch.cuda.current_stream() if stream is None else stream
+        s1, s2 = self.side
+        ev = self.ev
+        qkw = dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
+                   seed_rht=self.seed_rht, dev_status=self.dev_status)
+        gkw = dict(path=self.path, dev_status=self.dev_status)
+        ev["start"].record(s0)
+        s1.wait_event(ev["start"])
+        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, stream=s1, **qkw)
+        ev["g"].record(s1)
+        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, stream=s0, **qkw)
+        ev["x"].record(s0)
+        ufp4.quantize(W, rounding=ufp4.ROUND_RTNE, out_row=self.Wr, out_col=self.Wc, stream=s0, **qkw)
+        ev["w"].record(s0)
+        ufp4.gemm(self.Xr, self.Wr, out=self.Y, layout=ufp4.FWD_Y, workspace=self.workspaces[0], stream=s0, **gkw)
+        s1.wait_event(ev["w"])
+        ufp4.gemm(self.Gr, self.Wc, out=self.dX, layout=ufp4.BWD_DX, workspace=self.workspaces[1], stream=s1, **gkw)
+        ev["dx"].record(s1)
+        s2.wait_event(ev["g"])
+        s2.wait_event(ev["x"])
+        ufp4.gemm(self.Gc, self.Xc, out=self.dW, layout=ufp4.BWD_DW, workspace=self.workspaces[2], stream=s2, **gkw)
+        ev["dw"].record(s2)
+        if join:
+            self.join(s0)
+        return self.Y, self.dX, self.dW
+
+    def join(self, stream=None):
+        """Make the caller's stream wait for the side streams of the last step_overlapped()."""
+        if self.overlap:
+            s0 = torch.cuda.current_stream() if stream is None else stream
+            s0.wait_event(self.ev["dx"])
+            s0.wait_event(self.ev["dw"])
 
     @property
     def flops(self) -> int:
@@ -105,10 +151,15 @@ class Ufp4MoE:
         ufp4.gemm_grouped(self.Gr, self.Wc, self.offsets_dev, self.offsets_host, self.H, ufp4.BWD_DX, out=self.dX, **kw)
         ufp4.gemm_grouped(self.Gc, self.Xc, self.offsets_dev, self.offsets_host, self.F, ufp4.BWD_DW, out=self.dW, **kw)
 
-    def step(self, X, W, dY, stream=None):
+    overlap = False     # the grouped step runs its calls in sequence on one stream
+
+    def step(self, X, W, dY, stream=None, join: bool = True):
         self.quantize(X, W, dY, stream)
         self.gemms(stream)
         return self.Y, self.dX, self.dW
+
+    def join(self, stream=None):
+        pass
 
     @property
     def flops(self) -> int:
