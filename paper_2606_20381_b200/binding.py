@@ -16,7 +16,7 @@ ROUND_RTNE, ROUND_SR = 0, 1
 AXIS_ROW, AXIS_COL, AXIS_BOTH = 0, 1, 2
 SCALE_FP32, SCALE_POW2, SCALE_E4M3_TENSOR = 0, 1, 2
 FWD_Y, BWD_DX, BWD_DW = 0, 1, 2
-PATH_AUTO, PATH_EXACT, PATH_TENSOR, PATH_PROMOTE = 0, 1, 2, 3
+PATH_AUTO, PATH_EXACT, PATH_TENSOR, PATH_PROMOTE, PATH_SPLIT = 0, 1, 2, 3, 4
 DEV_NONFINITE, DEV_EXP_WINDOW, DEV_WAIT_TIMEOUT = 1, 2, 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -206,7 +206,7 @@ def gemm_launch_count(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:
 
 
 def gemm_path_name(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> str:
-    return {PATH_EXACT: "exact", PATH_TENSOR: "tensor", PATH_PROMOTE: "promote"}[gemm_path_taken(A, B, path)[0]]
+    return {PATH_EXACT: "exact", PATH_TENSOR: "tensor", PATH_PROMOTE: "promote", PATH_SPLIT: "split"}[gemm_path_taken(A, B, path)[0]]
 
 
 def _alloc_out(rows: int, cols: int, bf16: bool, device) -> torch.Tensor:

@@ -23,6 +23,12 @@ int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, i
                         int64_t M, int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n,
                         void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
+size_t gemm_split_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
+int gemm_split_kernel_launches();
+bool gemm_split_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
+int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int64_t M,
+                      int64_t N, int64_t K, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
 static int check_operand(const ufp4_qtensor *q) {
     if (!q || !q->codes || !q->scales) return UFP4_ERR_NULL;
     if (q->grid < 0 || q->grid > 2 || q->scale_fmt < 0 || q->scale_fmt > 2) return UFP4_ERR_ENUM;
@@ -38,7 +44,7 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                          int mode, int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                          int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                          void *stream) {
-    if (path < 0 || path > 3) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 4) return UFP4_ERR_ENUM;
     if (!C) return UFP4_ERR_NULL;
     if (ldc < N) return UFP4_ERR_SHAPE;
     if (!aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
@@ -53,7 +59,16 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                                       workspace, workspace_bytes, dev_status, stream);
         if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
     }
-    // PROMOTE, or AUTO for scale formats the folded path cannot take
+    // SPLIT, or AUTO for scale formats the folded path cannot take (plain products only)
+    const bool split_ok = gemm_split_supported(A, B, M, N, K, mode);
+    if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_SPLIT || (path == UFP4_PATH_AUTO && split_ok)) {
+        const size_t need = gemm_split_workspace_bytes(A->rows, B->rows, A->k);
+        if (workspace && workspace_bytes >= need)
+            return gemm_split_launch(A, B, C, ldc, c_is_bf16, M, N, K, workspace, workspace_bytes, dev_status, stream);
+        if (path == UFP4_PATH_SPLIT) return UFP4_ERR_WORKSPACE;
+    }
+    // PROMOTE, or AUTO for what neither tensor-core operand form can take
     {
         const size_t need = gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
         if (workspace && workspace_bytes >= need)
@@ -97,7 +112,12 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     const bool pow2 = A->scale_fmt == UFP4_SCALE_POW2 && B->scale_fmt == UFP4_SCALE_POW2;
     if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
         return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
-    return ufp4::gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
+    // AUTO may take SPLIT (plain products) or PROMOTE (grouped products): enough for either
+    const size_t split = ufp4::gemm_split_workspace_bytes(A->rows, B->rows, A->k);
+    const size_t promote = ufp4::gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
+    if (path == UFP4_PATH_SPLIT) return split;
+    if (path == UFP4_PATH_PROMOTE) return promote;
+    return split > promote ? split : promote;
 }
 
 extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B, int path, int *kernel_launches) {
@@ -105,15 +125,19 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (rc != UFP4_OK) return rc;
     rc = ufp4::check_operand(B);
     if (rc != UFP4_OK) return rc;
-    if (path < 0 || path > 3) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 4) return UFP4_ERR_ENUM;
     if (A->k != B->k) return UFP4_ERR_SHAPE;
     bool tensor_ok = ufp4::gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0);
+    bool split_ok = ufp4::gemm_split_supported(A, B, A->rows, B->rows, A->k, 0);
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
     int taken = path == UFP4_PATH_EXACT ? UFP4_PATH_EXACT
-              : (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) ? UFP4_PATH_TENSOR : UFP4_PATH_PROMOTE;
+              : (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) ? UFP4_PATH_TENSOR
+              : (path == UFP4_PATH_SPLIT || (path == UFP4_PATH_AUTO && split_ok)) ? UFP4_PATH_SPLIT : UFP4_PATH_PROMOTE;
     if (kernel_launches)
         *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : taken == UFP4_PATH_TENSOR ? ufp4::gemm_tensor_kernel_launches()
-                                                                                     : ufp4::gemm_promote_kernel_launches();
+                         : taken == UFP4_PATH_SPLIT ? ufp4::gemm_split_kernel_launches()
+                                                    : ufp4::gemm_promote_kernel_launches();
     return taken;
 }
 

@@ -22,7 +22,7 @@ def three_products(X, W, dY, grid, scale_fmt=oracle.SCALE_FP32, seed_rht=1, seed
     return {"fwd_y": (Xr, Wr, ufp4.FWD_Y), "bwd_dx": (Gr, Wc, ufp4.BWD_DX), "bwd_dw": (Gc, Xc, ufp4.BWD_DW)}
 
 
-@pytest.mark.parametrize("path", [ufp4.PATH_EXACT, ufp4.PATH_PROMOTE])
+@pytest.mark.parametrize("path", [ufp4.PATH_EXACT, ufp4.PATH_PROMOTE, ufp4.PATH_SPLIT])
 @pytest.mark.parametrize("grid", [oracle.GRID_INT4, oracle.GRID_E1M2, oracle.GRID_E2M1])
 def test_tiny_layer_all_three_products(grid, path):
     X, W, dY = inputs.tiny_layer(0)
@@ -38,7 +38,7 @@ def test_tiny_layer_all_three_products(grid, path):
     assert np.linalg.norm(got - exact) / np.linalg.norm(exact) < 0.2
 
 
-@pytest.mark.parametrize("path", [ufp4.PATH_EXACT, ufp4.PATH_PROMOTE])
+@pytest.mark.parametrize("path", [ufp4.PATH_EXACT, ufp4.PATH_PROMOTE, ufp4.PATH_SPLIT])
 @pytest.mark.parametrize("scale_fmt", [oracle.SCALE_FP32, oracle.SCALE_POW2, oracle.SCALE_E4M3_TENSOR])
 def test_ragged_shapes_and_scale_formats_exact_path(scale_fmt, path):
     M, N, K = 200, 72, 176
@@ -60,27 +60,30 @@ def test_ragged_shapes_and_scale_formats_exact_path(scale_fmt, path):
     assert torch.all(out[:, N:] == 7.0)
 
 
-@pytest.mark.parametrize("shape", [(130, 260, 144), (384, 512, 1040), (1, 1, 16), (128, 128, 4096), (1024, 1536, 2048)])
-def test_promote_path_shapes(shape):
-    """The tensor-core + promotion path for FP32 scales over ragged, multi-tile and long-K shapes."""
+@pytest.mark.parametrize("path", [ufp4.PATH_PROMOTE, ufp4.PATH_SPLIT])
+@pytest.mark.parametrize("shape", [(130, 260, 144), (384, 512, 1040), (1, 1, 16), (128, 128, 4096), (1024, 1536, 2048),
+                                   (2600, 1100, 528)])
+def test_fp32_scale_tensor_core_paths_shapes(shape, path):
+    """The two tensor-core paths for FP32 scales (block promotion; FP16 two-piece operands) over ragged, multi-tile and
+    long-K shapes; the last shape gives the persistent CTA pairs several tiles each."""
     M, N, K = shape
     X = inputs.heavy_tailed_activations(M, K, seed=21)
     W = inputs.normal_bf16(N, K, 0.02, seed=22)
     A = oracle_quantize(X, oracle.AXIS_ROW, rht_block=16, scale_fmt=oracle.SCALE_FP32, seed_rht=5)
     B = oracle_quantize(W, oracle.AXIS_ROW, rht_block=16, scale_fmt=oracle.SCALE_FP32, seed_rht=5)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    out = ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_PROMOTE, dev_status=status)
+    out = ufp4.gemm(to_device(A), to_device(B), path=path, dev_status=status)
     assert int(status.item()) == 0
     if M * N <= 1 << 19:
         ref, S = oracle.gemm(A, B)
-        assert_gemm_close(out.cpu().numpy(), ref, S, f"promote {shape}")
+        assert_gemm_close(out.cpu().numpy(), ref, S, f"path {path} {shape}")
     else:
         rng = np.random.default_rng(7)
         im, in_ = rng.integers(0, M, 20000), rng.integers(0, N, 20000)
         c, s = oracle.gemm_sampled(A, B, im, in_)
-        assert_gemm_close(out.cpu().numpy()[im, in_], c, s, f"promote sampled {shape}")
-    assert torch.equal(out, ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_PROMOTE))
-    assert ufp4.gemm_path_name(to_device(A), to_device(B), ufp4.PATH_AUTO) == "promote"
+        assert_gemm_close(out.cpu().numpy()[im, in_], c, s, f"path {path} sampled {shape}")
+    assert torch.equal(out, ufp4.gemm(to_device(A), to_device(B), path=path))
+    assert ufp4.gemm_path_name(to_device(A), to_device(B), ufp4.PATH_AUTO) == "split"
 
 
 def test_integer_and_one_hot_operands():

@@ -130,7 +130,7 @@ def test_grouped_products_small():
 
 
 @pytest.mark.parametrize("grid", [oracle.GRID_INT4, oracle.GRID_E1M2, oracle.GRID_E2M1])
-@pytest.mark.parametrize("path", [ufp4.PATH_TENSOR, ufp4.PATH_PROMOTE, ufp4.PATH_EXACT])
+@pytest.mark.parametrize("path", [ufp4.PATH_TENSOR, ufp4.PATH_PROMOTE, ufp4.PATH_SPLIT, ufp4.PATH_EXACT])
 def test_every_nibble_code_on_every_path(grid, path):
     """Hand-made operands holding all 16 nibble codes (also the ones the quantizer never emits: INT4 0x8 = -8, the
     negative zero of the sign | magnitude grids) with scales spread over the exponent window, zero scales included."""
