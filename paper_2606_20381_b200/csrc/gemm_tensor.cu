@@ -65,7 +65,11 @@ struct DecodeOperand {
 struct DecodeParams {
     DecodeOperand op[2];    // A and B in one launch
     int64_t K;
-    int64_t a_ctas;         // CTAs [0, a_ctas) work on A, the rest on B
+    int64_t a_ctas;         // CTAs [0, a_ctas) work on A, the next ones on B
+    int64_t tbl_cta;        // this CTA (if launched) lists the row tiles of a row-grouped product
+    const int64_t *offsets; // row offsets of the groups (device), num_groups + 1 of them
+    int num_groups;
+    int2 *mtiles;           // (first row, group) of every 256-row tile, group by group
     int32_t *dev_status;
 };
 
@@ -77,6 +81,14 @@ template <int TPR>
 __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const DecodeParams P) {
     __shared__ int s_emax[kDecodeThreads / 32];
     constexpr int kRowsPerCta = kDecodeThreads / TPR, kWarpsPerRow = TPR / 32;
+    if ((int64_t)blockIdx.x == P.tbl_cta) {
+        if (threadIdx.x == 0) {
+            int n = 0;
+            for (int g = 0; g < P.num_groups; ++g)
+                for (int64_t m = P.offsets[g]; m < P.offsets[g + 1]; m += 2 * kTM) P.mtiles[n++] = make_int2((int)m, g);
+        }
+        return;
+    }
     const bool is_b = (int64_t)blockIdx.x >= P.a_ctas;
     const DecodeOperand &O = P.op[is_b ? 1 : 0];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -325,11 +337,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int j = 0; j < 32; ++j) v[cur][j] = 0u;
                 }
                 const int64_t n_base = t.n0 + c * 32;
-                if (n_base >= P.N || c_row >= P.M) continue;     // warp-uniform: the whole box would be clipped
+                if (n_base >= P.N || c_row >= t.row_end) continue;     // warp-uniform: the whole box is clipped or not this tile's
                 if (n_base + 32 > P.N && P.n_unaligned) {
                     // The TMA clips in 16-byte units: a last chunk whose valid part does not end on a 16-byte boundary
                     // is written with plain predicated stores so that nothing right of column N is touched.
-                    if (m_own < P.M) {
+                    if (m_own < t.row_end) {
                         for (int j = 0; j < 32 && n_base + j < P.N; ++j) {
                             const float val = __uint_as_float(v[cur][j]) * ra * refb_s[(rbuf ^ 1) * kTN + c * 32 + j];
                             const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
@@ -419,9 +431,10 @@ static bool make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t K,
 
 static size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// decoded operands, reference vectors, and the row-tile list of a row-grouped product (at most one tile per 128 rows)
 size_t gemm_tensor_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K) {
     return round_up((size_t)a_rows * K, 256) + round_up((size_t)b_rows * K, 256) + round_up((size_t)a_rows * 4, 256) +
-           round_up((size_t)b_rows * 4, 256);
+           round_up((size_t)b_rows * 4, 256) + round_up((size_t)(a_rows / 128 + 2) * sizeof(int2), 256);
 }
 
 int gemm_tensor_kernel_launches() { return 2; }
@@ -438,7 +451,6 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
                        int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                        int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                        void *stream) {
-    (void)host_offsets;
     if (!aligned_to(workspace, 256)) return UFP4_ERR_ALIGN;
     if (workspace_bytes < gemm_tensor_workspace_bytes(A->rows, B->rows, K)) return UFP4_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -447,6 +459,16 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     uint8_t *B8 = A8 + round_up((size_t)A->rows * K, 256);
     float *refA = reinterpret_cast<float *>(B8 + round_up((size_t)B->rows * K, 256));
     float *refB = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(refA) + round_up((size_t)A->rows * 4, 256));
+    int2 *mtiles = reinterpret_cast<int2 *>(reinterpret_cast<uint8_t *>(refB) + round_up((size_t)B->rows * 4, 256));
+    // CTA pairs (cta_group::2), except for row-grouped products with a short reduction: those are bound by writing C, and
+    // single CTAs on 128-row tiles waste nothing on groups of 128 (mod 256) rows
+    const int cg = (mode == 1 && K < 4096) ? 1 : 2;
+    // row-grouped product on pairs: 256-row tiles group by group (the decode launch lists them from the device offsets)
+    int64_t row_tiles = 0;
+    if (mode == 1) {
+        if (A->rows > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
+        for (int g = 0; g < num_groups; ++g) row_tiles += (host_offsets[g + 1] - host_offsets[g] + 2 * kTM - 1) / (2 * kTM);
+    }
 
     DecodeParams D = {};
     D.op[0] = DecodeOperand{static_cast<const uint8_t *>(A->codes), static_cast<const float *>(A->scales),
@@ -459,7 +481,9 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     const int64_t rows_per_cta = kDecodeThreads / tpr;
     D.a_ctas = (A->rows + rows_per_cta - 1) / rows_per_cta;
     D.dev_status = dev_status;
-    const int64_t decode_ctas = D.a_ctas + (B->rows + rows_per_cta - 1) / rows_per_cta;
+    D.tbl_cta = D.a_ctas + (B->rows + rows_per_cta - 1) / rows_per_cta;
+    D.offsets = offsets; D.num_groups = num_groups; D.mtiles = mtiles;
+    const int64_t decode_ctas = D.tbl_cta + (mode == 1 && cg == 2 ? 1 : 0);
     if (decode_ctas > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     const unsigned dg = (unsigned)decode_ctas;
     if (tpr == 32) decode_rows_kernel<32><<<dg, kDecodeThreads, 0, st>>>(D);
@@ -468,8 +492,6 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     else decode_rows_kernel<256><<<dg, kDecodeThreads, 0, st>>>(D);
     if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
 
-    // CTA pairs (cta_group::2) wherever a 256-row output tile cannot straddle two row groups
-    const int cg = (mode == 1) ? 1 : 2;
     CUtensorMap tmA, tmB;
     if (!make_map(&tmA, A8, A->rows, K, kTM) || !make_map(&tmB, B8, B->rows, K, cg == 2 ? TcCfg<2>::kBRows : TcCfg<1>::kBRows))
         return UFP4_ERR_CUDA;
@@ -496,7 +518,8 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     P.M = M; P.N = N; P.K = K; P.mode = mode;
     P.offsets = offsets; P.num_groups = num_groups; P.group_n = group_n;
     P.refA = refA; P.refB = refB; P.dev_status = dev_status;
-    P.mt = (int)((M + kTM * cg - 1) / (kTM * cg));
+    P.mtiles = mtiles;
+    P.mt = (mode == 1 && cg == 2) ? (int)row_tiles : (int)((M + kTM * cg - 1) / (kTM * cg));
     P.nt = (int)((N + kTN - 1) / kTN);
     const int64_t total = (int64_t)P.mt * P.nt * (mode == 2 ? num_groups : 1);
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;

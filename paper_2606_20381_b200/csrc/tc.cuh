@@ -127,11 +127,15 @@ struct TcParams {
     int32_t *dev_status;
     int mt, nt, total_tiles;
     int n_unaligned;          // N * sizeof(element of C) is not a multiple of 16
+    // mode 1 on CTA pairs: the 256-row tiles are laid out group by group, so that a tile never straddles two groups;
+    // entry i = (first row, group) of row-tile i (a group of 128 (mod 256) rows ends with a half-filled tile)
+    const int2 *mtiles;
 };
 
 struct TileInfo {
     int64_t m0, n0, b_row0, c_row0;
     int kb0, nkb;
+    int64_t row_end;          // rows of C from here on are not this tile's to write
 };
 
 // Tile `tile` of the launch, as seen by the CTA of rank `rank` in its group of CG CTAs: the group owns a
@@ -149,7 +153,14 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile, int r
     t.c_row0 = 0;
     t.kb0 = 0;
     t.nkb = (int)((P.K + kTK - 1) / kTK);
-    if (P.mode == 1) {
+    t.row_end = P.M;
+    if (P.mode == 1 && CG == 2) {
+        const int2 e = P.mtiles[rem / P.nt];
+        t.m0 = (int64_t)e.x + (int64_t)rank * kTM;
+        t.b_row0 = (int64_t)e.y * P.group_n;
+        const int64_t group_end = P.offsets[e.y + 1];
+        t.row_end = group_end < (int64_t)e.x + 2 * kTM ? group_end : (int64_t)e.x + 2 * kTM;
+    } else if (P.mode == 1) {
         int lo = 0, hi = P.num_groups;
         while (hi - lo > 1) {
             int mid = (lo + hi) >> 1;

@@ -152,3 +152,23 @@ def test_every_nibble_code_on_every_path(grid, path):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert_gemm_close(out.cpu().numpy(), c_ref, s_ref, f"grid {grid} path {path}")
+
+
+def test_row_grouped_product_long_reduction_on_cta_pairs():
+    """Row-grouped products with K >= 4096 run on CTA pairs whose 256-row tiles are laid out group by group: groups of
+    128 (mod 256) rows (half-filled last tile), an empty group, a ragged N; every row must come from its own expert."""
+    offsets = [0, 128, 128, 512, 768, 1408]
+    E, H, F = 5, 4096, 200
+    X = inputs.heavy_tailed_activations(offsets[-1], H, seed=41)
+    W = inputs.normal_bf16(E * F, H, 0.02, seed=42)
+    kw = dict(rht_block=16, grid=oracle.GRID_INT4, seed_rht=1, scale_fmt=oracle.SCALE_POW2)
+    Xr = oracle_quantize(X, oracle.AXIS_ROW, **kw)
+    Wr = oracle_quantize(W, oracle.AXIS_ROW, **kw)
+    off_h = torch.tensor(offsets, dtype=torch.int64)
+    ref, S = grouped_reference(Xr, Wr, offsets, F, ufp4.FWD_Y)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.full((offsets[-1], F), 7.0, dtype=torch.float32, device="cuda")
+    ufp4.gemm_grouped(to_device(Xr), to_device(Wr), off_h.cuda(), off_h, F, ufp4.FWD_Y, path=ufp4.PATH_TENSOR,
+                      dev_status=status, out=out)
+    assert int(status.item()) == 0
+    assert_gemm_close(out.cpu().numpy(), ref, S, "row-grouped, pairs")
