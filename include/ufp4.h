@@ -152,7 +152,7 @@ int ufp4_selftest_division(int32_t *dev_mismatches, void *stream);
 size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path);
 
 /* GEMM paths (given a workspace of ufp4_gemm_workspace_bytes(A, B, path); without one AUTO falls back to EXACT).
- * AUTO:    TENSOR when both operands use POW2 scales, else SPLIT (plain products) or PROMOTE (grouped products).
+ * AUTO:    TENSOR when both operands use POW2 scales, else SPLIT.
  * EXACT:   CUDA-core kernel: integer block partials (dp4a) promoted with the two FP32 block scales, FP64 running sum;
  *          every grid and scale format, no workspace; the slow reference path.
  * TENSOR:  tcgen05 / TMEM kernel on 8-bit floating-point operands into which code x 2^e is folded exactly (POW2 scales
@@ -161,7 +161,7 @@ size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, i
  *          CUDA cores promote it with sA * sB into FP32 accumulators; every grid and scale format (Table 1's FP32 scales).
  * SPLIT:   tcgen05 / TMEM kernel on FP16 operands: each dequantized value, relative to a per-row power-of-two
  *          reference, is split into two FP16 pieces (22 significant bits) and the product taken by three MMAs per K
- *          step; every grid and scale format (Table 1's FP32 scales), plain products only; blocks more than 2^26 below
+ *          step; every grid and scale format (Table 1's FP32 scales), plain and grouped; blocks more than 2^26 below
  *          a row's largest scale are flushed and set UFP4_DEV_EXP_WINDOW. */
 typedef enum {
     UFP4_PATH_AUTO = 0, UFP4_PATH_EXACT = 1, UFP4_PATH_TENSOR = 2, UFP4_PATH_PROMOTE = 3, UFP4_PATH_SPLIT = 4

@@ -26,8 +26,9 @@ int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, i
 size_t gemm_split_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
 int gemm_split_kernel_launches();
 bool gemm_split_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
-int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int64_t M,
-                      int64_t N, int64_t K, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
+                      int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets, int num_groups,
+                      int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
 static int check_operand(const ufp4_qtensor *q) {
     if (!q || !q->codes || !q->scales) return UFP4_ERR_NULL;
@@ -59,13 +60,14 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                                       workspace, workspace_bytes, dev_status, stream);
         if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
     }
-    // SPLIT, or AUTO for scale formats the folded path cannot take (plain products only)
+    // SPLIT, or AUTO for scale formats the folded path cannot take
     const bool split_ok = gemm_split_supported(A, B, M, N, K, mode);
     if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_SPLIT || (path == UFP4_PATH_AUTO && split_ok)) {
         const size_t need = gemm_split_workspace_bytes(A->rows, B->rows, A->k);
         if (workspace && workspace_bytes >= need)
-            return gemm_split_launch(A, B, C, ldc, c_is_bf16, M, N, K, workspace, workspace_bytes, dev_status, stream);
+            return gemm_split_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
+                                     workspace, workspace_bytes, dev_status, stream);
         if (path == UFP4_PATH_SPLIT) return UFP4_ERR_WORKSPACE;
     }
     // PROMOTE, or AUTO for what neither tensor-core operand form can take

@@ -58,7 +58,11 @@ struct SDecodeOperand {
 struct SDecodeParams {
     SDecodeOperand op[2];   // A and B in one launch
     int64_t K;
-    int64_t a_ctas;         // CTAs [0, a_ctas) work on A, the rest on B
+    int64_t a_ctas;         // CTAs [0, a_ctas) work on A, the next ones on B
+    int64_t tbl_cta;        // this CTA (if launched) lists the row tiles of a row-grouped product
+    const int64_t *offsets; // row offsets of the groups (device), num_groups + 1 of them
+    int num_groups;
+    int2 *mtiles;           // (first row, group) of every 256-row tile, group by group
     int32_t *dev_status;
 };
 
@@ -85,6 +89,14 @@ template <int TPR>
 __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDecodeParams P) {
     __shared__ uint32_t s_max[kSDecodeThreads / 32];
     constexpr int kRowsPerCta = kSDecodeThreads / TPR, kWarpsPerRow = TPR / 32;
+    if ((int64_t)blockIdx.x == P.tbl_cta) {
+        if (threadIdx.x == 0) {
+            int n = 0;
+            for (int g = 0; g < P.num_groups; ++g)
+                for (int64_t m = P.offsets[g]; m < P.offsets[g + 1]; m += 2 * kTM) P.mtiles[n++] = make_int2((int)m, g);
+        }
+        return;
+    }
     const bool is_b = (int64_t)blockIdx.x >= P.a_ctas;
     const SDecodeOperand &O = P.op[is_b ? 1 : 0];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -220,7 +232,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
     const int group_id = blockIdx.x / 2, num_groups_launched = gridDim.x / 2;
     const uint32_t lead_full_bar = map_to_cta(full_bar, 0);
     const uint32_t lead_tempty_bar = map_to_cta(tempty_bar, 0);
-    const int nks = (int)((P.K + kSpK - 1) / kSpK);          // K steps of a tile
+    const int nks_all = (int)((P.K + kSpK - 1) / kSpK);      // K steps of a tile that reduces over all of K
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kSpStages; ++s) {
@@ -251,10 +263,13 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
-                const int32_t m0 = (tile / P.nt) * (2 * kTM) + rank * kTM, n0 = (tile % P.nt) * kTN + rank * (kTN / 2);
+                const TileInfo t = tile_info<2>(P, tile, rank);
+                const int32_t m0 = (int32_t)t.m0, n0 = (int32_t)(t.b_row0 + t.n0) + rank * (kTN / 2);
+                // tile_info counts the reduction in units of 128 elements; a K step here is 64
+                const int ks0 = 2 * t.kb0, nks = P.mode == 2 ? 2 * t.nkb : nks_all;
                 for (int ks = 0; ks < nks; ++ks) {
                     if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const int32_t kc = ks * kSpK;
+                    const int32_t kc = (ks0 + ks) * kSpK;
                     const uint32_t fb = lead_full_bar + 8 * stage, dst = base + stage * kSpStageBytes;
                     if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, kSpStageBytes);
                     else mbar_expect_tx_cluster(fb, kSpStageBytes);
@@ -273,6 +288,9 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+                const TileInfo t = tile_info<2>(P, tile, rank);
+                const int nks = P.mode == 2 ? 2 * t.nkb : nks_all;
+                if (nks == 0) continue;                       // empty group: the epilogue writes zeros
                 if (!mbar_wait(tempty_bar, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 for (int ks = 0; ks < nks; ++ks) {
@@ -309,46 +327,55 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
         uint32_t acc_phase = 0, rb_phase[2] = {0u, 0u};
         bool ok = true;
         for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
-            const int64_t m0 = (int64_t)(tile / P.nt) * (2 * kTM) + rank * kTM, n0 = (int64_t)(tile % P.nt) * kTN;
+            const TileInfo t = tile_info<2>(P, tile, rank);
+            const int64_t m0 = t.m0, n0 = t.n0;
+            const bool has_k = P.mode == 2 ? t.nkb > 0 : true;
             const int64_t m_own = m0 + q * 32 + lane;
             const float ra = m_own < P.M ? P.refA[m_own] : 0.0f;
             {
                 const int64_t n = n0 + et;
-                refb_s[rbuf * kTN + et] = n < P.N ? P.refB[n] : 0.0f;
+                refb_s[rbuf * kTN + et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
                 mbar_arrive(rb_bar + 8 * rbuf);
                 if (!mbar_wait(rb_bar + 8 * rbuf, rb_phase[rbuf], abort_flag)) { ok = false; break; }
                 rb_phase[rbuf] ^= 1u;
             }
             const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s + rbuf * kTN);
             rbuf ^= 1;
-            if (!mbar_wait(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            acc_phase ^= 1u;
+            if (has_k) {
+                if (!mbar_wait(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                acc_phase ^= 1u;
+            }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            const int32_t c_row = (int32_t)(m0 + q * 32);
+            const int32_t c_row = (int32_t)(m0 + q * 32), c_grp = (int32_t)(t.c_row0 / (P.M > 0 ? P.M : 1));
             uint32_t v0[32], v1[32];
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
                 const int c = 4 * half + cc;
-                tc_ld32(taddr + (uint32_t)(c * 32), v0);
-                tc_ld32(taddr + (uint32_t)(kTN + c * 32), v1);
-                tc_wait_ld();
-                if (cc == 3) {
+                if (has_k) {
+                    tc_ld32(taddr + (uint32_t)(c * 32), v0);
+                    tc_ld32(taddr + (uint32_t)(kTN + c * 32), v1);
+                    tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v0[j] = v1[j] = 0u;
+                }
+                if (has_k && cc == 3) {
                     // every column of both accumulators has been read: hand them back to the MMA warp
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(lead_tempty_bar);
                 }
                 const int64_t n_base = n0 + c * 32;
-                if (n_base >= P.N || c_row >= P.M) continue;     // warp-uniform: the whole box would be clipped
+                if (n_base >= P.N || c_row >= t.row_end) continue;   // warp-uniform: the box is clipped or not this tile's
                 if (n_base + 32 > P.N && P.n_unaligned) {
                     // The TMA clips in 16-byte units: a last chunk whose valid part does not end on a 16-byte boundary
                     // is written with plain predicated stores so that nothing right of column N is touched.
-                    if (m_own < P.M) {
+                    if (m_own < t.row_end) {
                         for (int j = 0; j < 32 && n_base + j < P.N; ++j) {
                             const float sum = __fmaf_rn(__uint_as_float(v1[j]), 1.0f / kSpLoScale, __uint_as_float(v0[j]));
                             const float val = sum * ra * refb_s[(rbuf ^ 1) * kTN + c * 32 + j];
-                            const int64_t idx = m_own * P.ldc + n_base + j;
+                            const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
                             if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(val);
                             else static_cast<float *>(P.C)[idx] = val;
                         }
@@ -390,8 +417,8 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                 __syncwarp();
                 if (lane == 0) {
                     asm volatile(
-                        "cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                        ::"l"(&tmC), "r"((int32_t)n_base), "r"(c_row), "r"(smem_u32(buf)) : "memory");
+                        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                        ::"l"(&tmC), "r"((int32_t)n_base), "r"(c_row), "r"(c_grp), "r"(smem_u32(buf)) : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
@@ -422,19 +449,19 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
 
 static size_t sp_round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// hi and lo FP16 arrays of both operands, then the two reference vectors
+// hi and lo FP16 arrays of both operands, the two reference vectors, and the row-tile list of a row-grouped product
 size_t gemm_split_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K) {
     return 2 * sp_round_up((size_t)a_rows * K * 2, 256) + 2 * sp_round_up((size_t)b_rows * K * 2, 256) +
-           sp_round_up((size_t)a_rows * 4, 256) + sp_round_up((size_t)b_rows * 4, 256);
+           sp_round_up((size_t)a_rows * 4, 256) + sp_round_up((size_t)b_rows * 4, 256) +
+           sp_round_up((size_t)(a_rows / 128 + 2) * sizeof(int2), 256);
 }
 
 int gemm_split_kernel_launches() { return 2; }
 
 bool gemm_split_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode) {
-    (void)A; (void)B;
-    if (mode != 0) return false;                        // grouped products take the promotion path
+    (void)mode;
     if (K % 16 != 0 || M < 1 || N < 1) return false;
-    if (M > 0x3FFFFFFF || N > 0x3FFFFFFF || K > 0x3FFFFFFF) return false;
+    if (A->rows > 0x3FFFFFFF || B->rows > 0x3FFFFFFF || K > 0x3FFFFFFF) return false;
     return true;
 }
 
@@ -450,8 +477,9 @@ static bool sp_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int64_t M,
-                      int64_t N, int64_t K, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
+int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
+                      int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets, int num_groups,
+                      int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
     if (!aligned_to(workspace, 256)) return UFP4_ERR_ALIGN;
     if (workspace_bytes < gemm_split_workspace_bytes(A->rows, B->rows, K)) return UFP4_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -461,6 +489,11 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
     __half *Bh = reinterpret_cast<__half *>(ws + 2 * a_bytes), *Bl = reinterpret_cast<__half *>(ws + 2 * a_bytes + b_bytes);
     float *refA = reinterpret_cast<float *>(ws + 2 * a_bytes + 2 * b_bytes);
     float *refB = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(refA) + sp_round_up((size_t)A->rows * 4, 256));
+    int2 *mtiles = reinterpret_cast<int2 *>(reinterpret_cast<uint8_t *>(refB) + sp_round_up((size_t)B->rows * 4, 256));
+    // row-grouped product: 256-row tiles group by group (the decode launch lists them from the device offsets)
+    int64_t row_tiles = 0;
+    if (mode == 1)
+        for (int g = 0; g < num_groups; ++g) row_tiles += (host_offsets[g + 1] - host_offsets[g] + 2 * kTM - 1) / (2 * kTM);
 
     SDecodeParams D = {};
     D.op[0] = SDecodeOperand{static_cast<const uint8_t *>(A->codes), A->scales, A->tensor_scale, A->ld_codes_bytes,
@@ -473,7 +506,9 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
     while (tpr < kSDecodeThreads && (K >> 4) >= (int64_t)16 * tpr) tpr *= 2;
     const int64_t rows_per_cta = kSDecodeThreads / tpr;
     D.a_ctas = (A->rows + rows_per_cta - 1) / rows_per_cta;
-    const int64_t decode_ctas = D.a_ctas + (B->rows + rows_per_cta - 1) / rows_per_cta;
+    D.tbl_cta = D.a_ctas + (B->rows + rows_per_cta - 1) / rows_per_cta;
+    D.offsets = offsets; D.num_groups = num_groups; D.mtiles = mtiles;
+    const int64_t decode_ctas = D.tbl_cta + (mode == 1 ? 1 : 0);
     if (decode_ctas > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     const unsigned dg = (unsigned)decode_ctas;
     if (tpr == 32) decode_split_kernel<32><<<dg, kSDecodeThreads, 0, st>>>(D);
@@ -489,12 +524,14 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
     {
         EncodeTiledFn fn = encode_tiled_fn();
         if (!fn) return UFP4_ERR_CUDA;
+        // C as [groups][rows][cols] so that the TMA store clips at the end of each group's rows and at N
+        const int64_t groups = mode == 2 ? num_groups : 1;
         const cuuint64_t es = c_is_bf16 ? 2 : 4;
-        cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-        cuuint64_t strides[1] = {(cuuint64_t)ldc * es};
-        cuuint32_t box[2] = {32, 32};
-        cuuint32_t estr[2] = {1, 1};
-        if (fn(&tmC, c_is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box,
+        cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)groups};
+        cuuint64_t strides[2] = {(cuuint64_t)ldc * es, (cuuint64_t)M * (cuuint64_t)ldc * es};
+        cuuint32_t box[3] = {32, 32, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        if (fn(&tmC, c_is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, C, dims, strides, box,
                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, c_is_bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return UFP4_ERR_CUDA;
@@ -502,11 +539,13 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
 
     TcParams P = {};
     P.C = C; P.ldc = ldc; P.c_is_bf16 = c_is_bf16;
-    P.M = M; P.N = N; P.K = K; P.mode = 0;
+    P.M = M; P.N = N; P.K = K; P.mode = mode;
+    P.offsets = offsets; P.num_groups = num_groups; P.group_n = group_n;
     P.refA = refA; P.refB = refB; P.dev_status = dev_status;
-    P.mt = (int)((M + 2 * kTM - 1) / (2 * kTM));
+    P.mtiles = mtiles;
+    P.mt = mode == 1 ? (int)row_tiles : (int)((M + 2 * kTM - 1) / (2 * kTM));
     P.nt = (int)((N + kTN - 1) / kTN);
-    const int64_t total = (int64_t)P.mt * P.nt;
+    const int64_t total = (int64_t)P.mt * P.nt * (mode == 2 ? num_groups : 1);
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;

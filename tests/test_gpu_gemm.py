@@ -139,7 +139,7 @@ def test_grouped_products_small():
     cases = {"fwd_y": (Xr, Wr, ufp4.FWD_Y, F), "bwd_dx": (Gr, Wc, ufp4.BWD_DX, H), "bwd_dw": (Gc, Xc, ufp4.BWD_DW, F)}
     for name, (A, B, layout, gn) in cases.items():
         ref, S = grouped_reference(A, B, offsets, gn, layout)
-        for path in (ufp4.PATH_EXACT, ufp4.PATH_PROMOTE):
+        for path in (ufp4.PATH_EXACT, ufp4.PATH_PROMOTE, ufp4.PATH_SPLIT):
             got = ufp4.gemm_grouped(to_device(A), to_device(B), off_d, off_h, gn, layout, path=path).cpu().numpy()
             assert got.shape == ref.shape, name
             assert_gemm_close(got, ref, S, f"grouped {name} path {path}")
