@@ -146,3 +146,30 @@ def test_grouped_products_small():
     # the empty group's dW is exactly zero
     got = ufp4.gemm_grouped(to_device(Gc), to_device(Xc), off_d, off_h, F, ufp4.BWD_DW, path=ufp4.PATH_EXACT)
     assert torch.all(got[F:2 * F] == 0)
+
+
+def test_split_path_exponent_window_and_extreme_scales():
+    """FP16 two-piece operands: block scales spanning 2^20 inside a row stay within the bound, a spread beyond the
+    window (2^26) is reported, and rows whose scales sit near the ends of the quantizer's range (2^-100, 2^100) work."""
+    M, N, K = 160, 272, 256
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    for b in range(K // 16):
+        x[:, 16 * b:16 * b + 16] *= 2.0 ** (-(b % 11) * 2)
+    x[3] *= 2.0 ** -90                           # tiny row: scales near 2^-100
+    x[5] *= 2.0 ** 100                           # huge row
+    w = rng.standard_normal((N, K)).astype(np.float32)
+    w[7] *= 2.0 ** -20                           # products stay inside FP32's range: 2^-110 .. 2^100
+    kw = dict(rht_block=16, scale_fmt=oracle.SCALE_FP32, seed_rht=1)
+    A = oracle_quantize(torch.from_numpy(x).bfloat16(), oracle.AXIS_ROW, **kw)
+    B = oracle_quantize(torch.from_numpy(w).bfloat16(), oracle.AXIS_ROW, grid=oracle.GRID_E1M2, **kw)
+    ref, S = oracle.gemm(A, B)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_SPLIT, dev_status=status)
+    assert int(status.item()) == 0
+    assert_gemm_close(out.cpu().numpy(), ref, S, "2^20 spread, extreme rows")
+    x[5] *= 2.0 ** -100
+    x[:, :16] *= 2.0 ** 30                       # one block 2^30 above the rest: the small blocks leave the window
+    A = oracle_quantize(torch.from_numpy(x).bfloat16(), oracle.AXIS_ROW, **kw)
+    ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_SPLIT, dev_status=status)
+    assert int(status.item()) & ufp4.DEV_EXP_WINDOW
