@@ -196,6 +196,24 @@ int ufp4_gemm_grouped(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
                       void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
 /*
+ * Tensor diagnostics of Sec. 3 on a BF16 matrix x [rows][cols] and its row variant q_row (FP32 or POW2 scales), with
+ * x' = x H'_16 per 16-block for rht_block == 16 (the quantizer's FP32 butterflies) or x' = x for rht_block == 0, and
+ * xq = level * scale.  dev_out (device, 19 doubles) receives
+ *   [0] sum x'^2   [1] sum (xq - x')^2   [2] sum xq x'      -> alpha = [2] / [0] (Eq. 3), NMSE = [1] / [0] (Sec. 3.3;
+ *                                                              Delta SQNR of Eq. 7 is 10 log10 of the ratio of two NMSEs)
+ *   [3 + i]  number of elements whose code has magnitude level i, i = 0..7 -> p_i of Eq. 6 (effective bucket ratio)
+ *   [11 + i] sum over those elements of (level_i - |x'| / s) in grid units -> Sec. 3.1's E[rho_G(t) - t] per bin
+ *            (elements of zero-scale blocks are counted in [3 + i] but add nothing here)
+ * The three sums of squares are FP32 inside a 16-block and FP64 across blocks (relative error below 1e-6), the
+ * per-level error sums FP32 per thread and FP64 across threads; everything is added in a fixed order: the result is
+ * reproducible.  workspace >= ufp4_diagnose_workspace_bytes(rows, cols) bytes of device memory.
+ * Not on the training hot path: a measurement pass (one read of x, codes and scales).
+ */
+size_t ufp4_diagnose_workspace_bytes(int64_t rows, int64_t cols);
+int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t ld, const ufp4_qtensor *q_row, int rht_block,
+                  uint64_t seed_rht, double *dev_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * ufp4_gemm without any device allocation by anyone (the paper has no counterpart to this entry point; it exists for
  * the library's users).  Some callers cannot provide the workspace ufp4_gemm's tensor-core path needs: a process
  * whose device memory has all been handed to a framework's pool, or code running at a point where calling cudaMalloc

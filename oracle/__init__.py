@@ -63,6 +63,10 @@ def lib():
         L.orc_gemm_sampled.argtypes = [p, p, i32, i32, f32, p, p, i32, i32, f32, i64, i64, i64, i64, p, p, p, p]
         L.orc_bin_bias.restype = None
         L.orc_bin_bias.argtypes = [p, p, i64, i32, p, p]
+        L.orc_diagnose.restype = None
+        L.orc_diagnose.argtypes = [p, i64, i64, i64, p, i64, p, i64, i32, i32, C.c_uint32, p]
+        L.orc_b_eff.restype = f64
+        L.orc_b_eff.argtypes = [p]
         _lib = L
     return _lib
 
@@ -214,3 +218,28 @@ def bin_bias(y: np.ndarray, codes: np.ndarray, grid: int):
     with np.errstate(invalid="ignore", divide="ignore"):
         mean = np.where(count > 0, total / np.maximum(count, 1), np.nan)
     return count, mean
+
+
+def diagnose(x_u16: np.ndarray, q: QTensor, rht_block: int, seed_rht: int) -> dict:
+    """Tensor diagnostics of the row variant q of the BF16 matrix x (Eq. 3, Eq. 6, Eq. 7 ingredients, Sec. 3.1 bias):
+    alpha, nmse, b_eff, count[8], bias[8] (mean of level - t per magnitude level, NaN where a level is unused)."""
+    x = np.ascontiguousarray(x_u16, dtype=np.uint16)
+    rows, cols = x.shape
+    assert q.scale_fmt != SCALE_E4M3_TENSOR and q.codes.shape == (rows, cols // 2)
+    codes = np.ascontiguousarray(q.codes, dtype=np.uint8)
+    scales = np.ascontiguousarray(q.scales, dtype=np.float32)
+    out = np.zeros(19, dtype=np.float64)
+    lib().orc_diagnose(_ptr(x), rows, cols, cols, _ptr(codes), cols // 2, _ptr(scales), cols // 16, q.grid, rht_block,
+                       int(rht_sign_mask(seed_rht)), _ptr(out))
+    return diagnostics_from_sums(out)
+
+
+def diagnostics_from_sums(out: np.ndarray) -> dict:
+    """alpha (Eq. 3), NMSE (Sec. 3.3), B_eff (Eq. 6) and the per-level bias from the 19 raw sums of orc_diagnose."""
+    count, bias_sum = out[3:11], out[11:19]
+    with np.errstate(invalid="ignore", divide="ignore"):
+        bias = np.where(count > 0, bias_sum / np.maximum(count, 1), np.nan)
+        alpha = out[2] / out[0] if out[0] > 0 else float("nan")
+        nmse = out[1] / out[0] if out[0] > 0 else float("nan")
+    return {"alpha": float(alpha), "nmse": float(nmse), "b_eff": float(lib().orc_b_eff(_ptr(np.ascontiguousarray(count)))),
+            "count": count.astype(np.int64), "bias": bias, "sums": out.copy()}

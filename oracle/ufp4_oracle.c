@@ -399,3 +399,57 @@ void orc_bin_bias(const float *y, const uint8_t *codes, int64_t n, int grid, int
         sum[idx] += mag - fabs((double)y[e]);
     }
 }
+
+/* ---------------------------------------------------------------- tensor diagnostics (Sec. 3.2 Eq. 3, Sec. 3.3 Eq. 6-7) */
+
+/* For the row variant (codes, FP32 scales) of the BF16 matrix x [rows][cols], with x' = x H'_16 per 16-block
+ * (rht_block == 16; FP32 butterflies as in the quantizer) or x' = x (rht_block == 0) and xq = level * scale:
+ *   out[0] = sum x'^2, out[1] = sum (xq - x')^2, out[2] = sum xq x'            (Eq. 3: alpha = out[2] / out[0];
+ *                                                                               Sec. 3.3: NMSE = out[1] / out[0])
+ *   out[3 + i]  = number of elements whose code has magnitude level i           (Eq. 6: p_i = out[3 + i] / n)
+ *   out[11 + i] = sum over those elements of (level_i - |x'| / s), grid units   (Sec. 3.1 per-bin bias; a zero-scale
+ *                                                                               block contributes 0 to it)
+ * All sums in FP64, elements in storage order. */
+void orc_diagnose(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, const uint8_t *codes, int64_t ld_codes,
+                  const float *scales, int64_t ld_scales, int grid, int rht_block, uint32_t sign_mask, double out[19]) {
+    const double *L = levels_of(grid);
+    for (int i = 0; i < 19; ++i) out[i] = 0.0;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t b = 0; b < cols / 16; ++b) {
+            float v[16];
+            for (int i = 0; i < 16; ++i) {
+                uint32_t bits = (uint32_t)x[r * ld + 16 * b + i] << 16;
+                memcpy(&v[i], &bits, 4);
+            }
+            if (rht_block == 16) orc_rht16_f32(v, sign_mask);
+            const double s = (double)scales[r * ld_scales + b];
+            for (int i = 0; i < 16; ++i) {
+                const int64_t e = 16 * b + i;
+                const uint8_t byte = codes[r * ld_codes + e / 2];
+                const int nibble = (e & 1) ? (byte >> 4) : (byte & 0xF);
+                const double val = orc_nibble_value(grid, nibble);
+                const double xp = (double)v[i], xq = val * s;
+                out[0] += xp * xp;
+                out[1] += (xq - xp) * (xq - xp);
+                out[2] += xq * xp;
+                int idx = 0;
+                for (int k = 0; k < 8; ++k)
+                    if (L[k] == fabs(val)) idx = k;
+                out[3 + idx] += 1.0;
+                if (s > 0.0) out[11 + idx] += fabs(val) - fabs(xp) / s;
+            }
+        }
+}
+
+/* Effective bucket ratio of Eq. 6 from the eight level counts: exp(-sum p_i log(p_i + eps)) / 8, natural log,
+ * eps = 1e-12 (the paper leaves eps and the base open). */
+double orc_b_eff(const double count[8]) {
+    double n = 0.0, ent = 0.0;
+    for (int i = 0; i < 8; ++i) n += count[i];
+    if (n <= 0.0) return 0.0;
+    for (int i = 0; i < 8; ++i) {
+        double p = count[i] / n;
+        ent -= p * log(p + 1e-12);
+    }
+    return exp(ent) / 8.0;
+}

@@ -24,7 +24,7 @@ LIB_PATH = os.path.join(_HERE, "libufp4.so")
 
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_qtensor_bytes", "ufp4_quantize",
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
-           "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes"]
+           "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes"]
 
 
 class _QTensorStruct(C.Structure):
@@ -72,6 +72,10 @@ def lib():
         L.ufp4_gemm_noalloc.argtypes = [qp, qp, vp, i64, i32, vp, vp]
         L.ufp4_gemm_noalloc_max_scratch_bytes.restype = sz
         L.ufp4_gemm_noalloc_max_scratch_bytes.argtypes = []
+        L.ufp4_diagnose_workspace_bytes.restype = sz
+        L.ufp4_diagnose_workspace_bytes.argtypes = [i64, i64]
+        L.ufp4_diagnose.restype = i32
+        L.ufp4_diagnose.argtypes = [vp, i64, i64, i64, qp, i32, u64, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -185,6 +189,18 @@ def selftest_division(stream=None) -> int:
     n = torch.zeros(1, dtype=torch.int32, device="cuda")
     _check(lib().ufp4_selftest_division(n.data_ptr(), _stream_ptr(stream)))
     return int(n.item())
+
+
+def diagnose(x: torch.Tensor, q_row: QTensor, rht_block: int = 16, seed_rht: int = 0, stream=None) -> torch.Tensor:
+    """ufp4_diagnose: the 19 raw sums (device, float64) for the BF16 matrix x and its row variant q_row."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    out = torch.empty(19, dtype=torch.float64, device=x.device)
+    ws = torch.empty(lib().ufp4_diagnose_workspace_bytes(rows, cols), dtype=torch.uint8, device=x.device)
+    s = q_row.struct()
+    _check(lib().ufp4_diagnose(x.data_ptr(), rows, cols, x.stride(0), C.byref(s), rht_block, seed_rht, out.data_ptr(),
+                               ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
+    return out
 
 
 def gemm_workspace_bytes(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:

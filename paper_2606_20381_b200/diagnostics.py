@@ -1,45 +1,34 @@
-"""Measurement helpers (plain torch ops on the GPU, not part of the hot path): the Shrinkage-Bias diagnostic of
-Sec. 3.1, b_G = E[rho_G(t) - t] restricted to the bin of each level, evaluated on a tensor quantized by libufp4."""
+"""Measurement helpers around ufp4_diagnose (not part of the hot path): the Shrinkage-Bias diagnostic of Sec. 3.1,
+b_G = E[rho_G(t) - t] restricted to the bin of each level, the operand projection alpha of Eq. 3, the NMSE behind
+Eq. 7 and the effective bucket ratio of Eq. 6, for a tensor quantized by libufp4.  The sums come from the library's
+kernel; this module only turns them into ratios."""
 from __future__ import annotations
+
+import math
 
 import torch
 
 from . import binding as ufp4
 
-_LEVELS = {ufp4.GRID_INT4: [0, 1, 2, 3, 4, 5, 6, 7], ufp4.GRID_E1M2: [0, .25, .5, .75, 1, 1.25, 1.5, 1.75],
-           ufp4.GRID_E2M1: [0, .5, 1, 1.5, 2, 3, 4, 6]}
 
-
-def hadamard16(device) -> torch.Tensor:
-    h = torch.ones(1, 1, dtype=torch.float64, device=device)
-    for _ in range(4):
-        h = torch.cat([torch.cat([h, h], 1), torch.cat([h, -h], 1)], 0)
-    return h / 4.0
-
-
-def unpack_levels(q: ufp4.QTensor) -> torch.Tensor:
-    """Magnitude level index (0..7) of every element of a quantized tensor, [rows][k]."""
-    c = q.packed_codes()
-    nib = torch.stack([c & 0xF, c >> 4], -1).reshape(c.shape[0], -1).to(torch.int16)
-    if q.grid == ufp4.GRID_INT4:
-        return torch.where(nib >= 8, 16 - nib, nib)
-    return nib & 7
+def tensor_diagnostics(x: torch.Tensor, q_row: ufp4.QTensor, rht_block: int, seed_rht: int) -> dict:
+    """alpha (Eq. 3), nmse (Sec. 3.3), b_eff (Eq. 6: natural log, eps = 1e-12, K = 8 magnitude buckets incl. zero),
+    count[8] and bias[8] (mean of level - t per magnitude level, NaN where a level is unused) of the row variant."""
+    sums = ufp4.diagnose(x, q_row, rht_block, seed_rht).cpu()
+    count, bias_sum = sums[3:11], sums[11:19]
+    n = float(count.sum())
+    ent = -sum((float(c) / n) * math.log(float(c) / n + 1e-12) for c in count) if n > 0 else 0.0
+    sxx = float(sums[0])
+    return {"alpha": float(sums[2]) / sxx if sxx > 0 else float("nan"),
+            "nmse": float(sums[1]) / sxx if sxx > 0 else float("nan"),
+            "b_eff": math.exp(ent) / 8.0,
+            "count": count.to(torch.int64),
+            "bias": torch.where(count > 0, bias_sum / count.clamp_min(1), torch.full_like(bias_sum, float("nan"))),
+            "sums": sums}
 
 
 def per_bin_bias(x: torch.Tensor, q_row: ufp4.QTensor, rht_block: int, seed_rht: int):
     """(count[8], mean of level - t per level) for the row variant q_row of the BF16 matrix x, t = |x'| / s in grid
-    units, x' the rotated input (FP64 matrix product with H'_16; a measurement, not a bit-exact replay)."""
-    rows, cols = x.shape
-    xb = x.double().reshape(rows, cols // 16, 16)
-    if rht_block == 16:
-        mask = ufp4.rht_sign_mask(seed_rht)
-        eps = torch.tensor([-1.0 if (mask >> i) & 1 else 1.0 for i in range(16)], dtype=torch.float64, device=x.device)
-        xb = (xb * eps) @ hadamard16(x.device)
-    s = q_row.scales.double().unsqueeze(-1)
-    t = torch.where(s > 0, xb.abs() / s.clamp_min(1e-300), torch.zeros_like(xb)).reshape(rows, cols)
-    idx = unpack_levels(q_row).long()
-    lv = torch.tensor(_LEVELS[q_row.grid], dtype=torch.float64, device=x.device)
-    err = lv[idx] - t
-    count = torch.bincount(idx.reshape(-1), minlength=8)
-    total = torch.zeros(8, dtype=torch.float64, device=x.device).index_add_(0, idx.reshape(-1), err.reshape(-1))
-    return count.cpu(), (total / count.clamp_min(1)).cpu()
+    units, x' the rotated input."""
+    d = tensor_diagnostics(x, q_row, rht_block, seed_rht)
+    return d["count"], d["bias"]

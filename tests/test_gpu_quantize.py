@@ -155,19 +155,29 @@ def test_division_shortcuts_match_ieee_division_exhaustively():
     assert ufp4.selftest_division() == 0
 
 
-def test_per_bin_bias_measurement_agrees_with_the_oracle():
-    """The Shrinkage-Bias measurement used by the quantizer sweep (torch ops on the CUDA quantizer's output) against the
-    oracle's per-bin bias on the same tensor: the uniform grid is unbiased on interior levels, E2M1 is not."""
+def test_tensor_diagnostics_agree_with_the_oracle():
+    """ufp4_diagnose (alpha of Eq. 3, NMSE of Sec. 3.3 / Eq. 7, level counts of Eq. 6, per-bin bias of Sec. 3.1) on the
+    CUDA quantizer's output against the oracle's sums on the same tensor; ragged sizes; reproducible."""
     from paper_2606_20381_b200 import diagnostics
-    x = inputs.spiky_normal(512, 1024, seed=3)
-    for grid in (ufp4.GRID_INT4, ufp4.GRID_E2M1):
+    x = inputs.spiky_normal(520, 1040, seed=3)
+    xb = inputs.bf16_bits(x)
+    for grid in (ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1):
         for rht in (0, 16):
             row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=rht, grid=grid, seed_rht=1)
-            count, bias = diagnostics.per_bin_bias(x.cuda(), row, rht, 1)
-            ref = oracle_quantize(x, oracle.AXIS_ROW, rht_block=rht, grid=grid, seed_rht=1, want_y=True)
-            rc, rb = oracle.bin_bias(ref.y, ref.codes, grid)
-            assert np.array_equal(count.numpy(), rc)
-            assert np.allclose(bias.numpy(), rb, atol=2e-5, equal_nan=True)
+            got = diagnostics.tensor_diagnostics(x.cuda(), row, rht, 1)
+            ref_q = oracle_quantize(x, oracle.AXIS_ROW, rht_block=rht, grid=grid, seed_rht=1, want_y=True)
+            ref = oracle.diagnose(xb, ref_q, rht, 1)
+            assert np.array_equal(got["count"].numpy(), ref["count"])
+            assert np.allclose(got["sums"].numpy()[:3], ref["sums"][:3], rtol=1e-6)   # FP32 inside a block, FP64 across
+            assert np.allclose(got["bias"].numpy(), ref["bias"], atol=2e-5, equal_nan=True)
+            assert abs(got["alpha"] - ref["alpha"]) < 1e-6 and abs(got["nmse"] - ref["nmse"]) < 1e-6 * ref["nmse"] + 1e-9
+            assert abs(got["b_eff"] - ref["b_eff"]) < 1e-12
+            # the older per-element measurement (oracle's y) gives the same per-bin means
+            rc, rb = oracle.bin_bias(ref_q.y, ref_q.codes, grid)
+            assert np.array_equal(got["count"].numpy(), rc)
+            assert np.allclose(got["bias"].numpy(), rb, atol=2e-5, equal_nan=True)
+            again = diagnostics.tensor_diagnostics(x.cuda(), row, rht, 1)
+            assert torch.equal(again["sums"], got["sums"])
     # direction of the effect the paper describes: after RHT the E2M1 levels 2 and 4 shrink, the uniform grid does not
     row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_E2M1, seed_rht=1)
     _, b = diagnostics.per_bin_bias(x.cuda(), row, 16, 1)
@@ -175,3 +185,19 @@ def test_per_bin_bias_measurement_agrees_with_the_oracle():
     row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_INT4, seed_rht=1)
     _, b = diagnostics.per_bin_bias(x.cuda(), row, 16, 1)
     assert abs(b[1:7]).max() < 0.05     # what remains is the decreasing density inside symmetric bins, not geometry
+
+
+def test_rht_helps_the_uniform_grid_more_than_e2m1_on_outlier_heavy_tensors():
+    """Sec. 3.3's observation on synthetic heavy-tailed activations: the RHT raises the effective bucket ratio of both
+    grids, and its SQNR change (Eq. 7) is better for the uniform grid than for E2M1."""
+    from paper_2606_20381_b200 import diagnostics
+    x = inputs.heavy_tailed_activations(2048, 2048, seed=9).cuda()
+    d = {}
+    for grid in (ufp4.GRID_INT4, ufp4.GRID_E2M1):
+        for rht in (0, 16):
+            row, _ = ufp4.quantize(x, axis=ufp4.AXIS_ROW, rht_block=rht, grid=grid, seed_rht=1)
+            d[(grid, rht)] = diagnostics.tensor_diagnostics(x, row, rht, 1)
+    dsqnr = {g: 10 * np.log10(d[(g, 0)]["nmse"] / d[(g, 16)]["nmse"]) for g in (ufp4.GRID_INT4, ufp4.GRID_E2M1)}
+    assert d[(ufp4.GRID_INT4, 16)]["b_eff"] > d[(ufp4.GRID_INT4, 0)]["b_eff"]
+    assert d[(ufp4.GRID_E2M1, 16)]["b_eff"] > d[(ufp4.GRID_E2M1, 0)]["b_eff"]
+    assert dsqnr[ufp4.GRID_INT4] > 0 and dsqnr[ufp4.GRID_INT4] > dsqnr[ufp4.GRID_E2M1]

@@ -515,3 +515,68 @@ def test_freivalds_and_closeness_to_the_unquantized_product():
     assert oracle.rht_sign_mask(1) != oracle.rht_sign_mask(5)
     Cm, _ = oracle.gemm(A, B)
     assert np.linalg.norm(Cm - exact) / np.linalg.norm(exact) > 0.5
+
+
+# ------------------------------------------------------------------ tensor diagnostics (Eq. 3, Eq. 6, Eq. 7)
+
+def test_effective_bucket_ratio_spans_one_over_k_to_one():
+    """Eq. 6: B_eff = exp(entropy) / K is 1/K when one bucket holds everything and 1 for uniform use of the K = 8 buckets."""
+    one = np.zeros(8)
+    one[3] = 1000.0
+    assert abs(oracle.diagnostics_from_sums(np.concatenate([[1, 0, 0], one, np.zeros(8)]))["b_eff"] - 1 / 8) < 1e-9
+    flat = np.full(8, 125.0)
+    assert abs(oracle.diagnostics_from_sums(np.concatenate([[1, 0, 0], flat, np.zeros(8)]))["b_eff"] - 1.0) < 1e-9
+    two = np.zeros(8)
+    two[[0, 5]] = 500.0                                     # two equally used buckets: exp(log 2) / 8
+    assert abs(oracle.diagnostics_from_sums(np.concatenate([[1, 0, 0], two, np.zeros(8)]))["b_eff"] - 2 / 8) < 1e-9
+
+
+@pytest.mark.parametrize("grid", [GRID_INT4, GRID_E1M2, GRID_E2M1])
+def test_diagnostics_of_exactly_representable_and_of_zero_tensors(grid):
+    """A tensor that lies on the grid quantizes without error: NMSE = 0, alpha = 1 (Eq. 3), zero bias in every bin; an
+    all-zero tensor uses one bucket (B_eff = 1/8)."""
+    rng = np.random.default_rng(5)
+    L = oracle.levels(grid)
+    idx = rng.integers(0, 8, size=(32, 64))
+    idx[:, ::16] = 7                                        # every block holds g_max, so its scale is a power of two
+    x = L[idx] * rng.choice([-1.0, 1.0], size=idx.shape) * 2.0 ** rng.integers(-3, 4, size=(32, 1))
+    xb = bf16_bits(x)
+    q = oracle.quantize(xb, AXIS_ROW, rht_block=0, grid=grid)
+    d = oracle.diagnose(xb, q, 0, 0)
+    assert d["nmse"] == 0.0 and d["alpha"] == 1.0
+    assert np.all(np.nan_to_num(d["bias"]) == 0.0)
+    assert np.array_equal(d["count"], np.bincount(idx.reshape(-1), minlength=8))
+    z = np.zeros((16, 32), dtype=np.uint16)
+    dz = oracle.diagnose(z, oracle.quantize(z, AXIS_ROW, rht_block=16, grid=grid, seed_rht=3), 16, 3)
+    assert abs(dz["b_eff"] - 1 / 8) < 1e-9 and dz["count"][0] == 16 * 32
+
+
+def test_diagnostics_against_a_matrix_formulation():
+    """The same sums from independent ingredients: x' by an FP64 matrix product with H'_16, xq by the dequantizer; the
+    residual of the projection is orthogonal to x' (Eq. 3), and quantization noise on a uniform grid with unit scale has
+    variance 1/12 per element."""
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((48, 160)) * np.exp(rng.standard_normal((48, 1)))
+    xb = bf16_bits(x)
+    mask = oracle.rht_sign_mask(7)
+    eps = np.array([-1.0 if (mask >> i) & 1 else 1.0 for i in range(16)])
+    Hp = np.diag(eps) @ oracle.hadamard_matrix(16)
+    for grid in (GRID_INT4, GRID_E2M1):
+        q = oracle.quantize(xb, AXIS_ROW, rht_block=16, grid=grid, seed_rht=7)
+        d = oracle.diagnose(xb, q, 16, 7)
+        xp = (bf16_vals(xb).reshape(48, 10, 16) @ Hp).reshape(48, 160)
+        xq = oracle.dequantize(q)
+        assert np.isclose(d["sums"][0], np.sum(xp * xp), rtol=1e-6)
+        assert np.isclose(d["nmse"], np.sum((xq - xp) ** 2) / np.sum(xp * xp), rtol=1e-4)
+        assert np.isclose(d["alpha"], np.sum(xq * xp) / np.sum(xp * xp), rtol=1e-6)
+        assert abs(np.sum((xq - d["alpha"] * xp) * xp)) < 1e-6 * np.sum(xp * xp)
+    # unit-scale uniform grid: every block holds 7 (scale exactly 1), the other elements are uniform in (-7, 7)
+    u = rng.uniform(-7, 7, size=(256, 256))
+    u[:, ::16] = 7.0
+    ub = bf16_bits(u)
+    q = oracle.quantize(ub, AXIS_ROW, rht_block=0, grid=GRID_INT4)
+    assert np.all(q.scales == 1.0)
+    d = oracle.diagnose(ub, q, 0, 0)
+    n_free = 256 * 256 * 15 / 16
+    assert abs(d["sums"][1] / n_free - 1 / 12) < 0.003      # BF16 inputs are themselves on a fine grid: still 1/12
+    assert np.nanmax(np.abs(d["bias"][1:7])) < 0.01         # symmetric bins: no bias (Sec. 3.1)
