@@ -16,6 +16,8 @@
  *   orc_dequantize        Sec. 2.1, "Q_G(T) ... denotes the dequantized numerical tensor"
  *   orc_gemm_f64          Sec. 2.2, Y^ = Q_G(X H') Q_G(W H')^T as a plain FP64 triple loop
  *   orc_bin_bias          Sec. 3.1, b_G = E[rho_G(t) - t] restricted to the bin of each level
+ *   orc_diagnose          Sec. 3.2 Eq. 3 (operand projection alpha), Sec. 3.3 (NMSE, Eq. 7) and Eq. 6 (level counts
+ *                         behind the effective bucket ratio, orc_b_eff), plus the per-bin bias sums again
  *
  * Readings taken where the paper is silent (each is restated in the repository's design notes):
  *   - E1M2 levels are {0,...,7}/4 (g_max 1.75); INT4 is the symmetric integer grid {-7..7} (g_max 7); both are the
