@@ -36,7 +36,8 @@ constexpr int kSpThreads = 64 + 32 * kSpEpiWarps;      // warp 0: TMA, warp 1: M
 constexpr int kSpEpiBufBytes = 32 * 128;
 constexpr int kSpOffEpi = kSpRing;
 constexpr int kSpOffRefB = kSpOffEpi + kSpEpiWarps * kSpEpiBufBytes;
-constexpr int kSpOffBars = kSpOffRefB + 2 * kTN * 4;
+constexpr int kSpOffBars = kSpOffRefB + kTN * 4;         // one refB buffer: with it, a decode CTA (no shared memory, 64
+                                                         // registers) fits on the SM beside this kernel's CTA
 constexpr int kSpSmem = kSpOffBars + 256;
 constexpr float kSpLoScale = 2048.0f;                 // 2^11
 constexpr int kSpFlushExp = -15;                      // blocks whose normalised scale is below 2^-15 are flushed
@@ -87,8 +88,7 @@ __device__ __forceinline__ void pow2_factors(int p, float *f1, float *f2) {
 // A CTA decodes 256 / TPR rows with TPR threads (32..256) on each (more threads on long rows: no idle tail).
 template <int TPR>
 __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDecodeParams P) {
-    __shared__ uint32_t s_max[kSDecodeThreads / 32];
-    constexpr int kRowsPerCta = kSDecodeThreads / TPR, kWarpsPerRow = TPR / 32;
+    constexpr int kRowsPerCta = kSDecodeThreads / TPR;
     if ((int64_t)blockIdx.x == P.tbl_cta) {
         if (threadIdx.x == 0) {
             int n = 0;
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
     }
     const bool is_b = (int64_t)blockIdx.x >= P.a_ctas;
     const SDecodeOperand &O = P.op[is_b ? 1 : 0];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
     const int t = threadIdx.x % TPR;
     const int64_t row = ((int64_t)blockIdx.x - (is_b ? P.a_ctas : 0)) * kRowsPerCta + threadIdx.x / TPR;
     const bool active = row < O.rows;
@@ -110,28 +110,23 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
                            ? static_cast<const void *>(static_cast<const uint8_t *>(O.scales) + r_safe * O.lds)
                            : static_cast<const void *>(static_cast<const float *>(O.scales) + r_safe * O.lds);
 
-    // largest block scale of the row (scales are non-negative: their bit patterns order like their values)
+    // largest block scale of the row (scales are non-negative: their bit patterns order like their values).  Every warp
+    // of a row scans the whole row's scales (the repeats hit in cache): no shared memory and no CTA barrier, so that
+    // this kernel's CTAs fit beside a resident product-kernel CTA on the same SM.
     uint32_t smax = 0u;
     if (active) {
-        int kb = t;
-        for (; kb + 7 * TPR < nkb; kb += 8 * TPR) {
+        int kb = lane;
+        for (; kb + 7 * 32 < nkb; kb += 8 * 32) {
             float s[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) s[u] = split_scale_of(O, srow, kb + u * TPR, ts);
+            for (int u = 0; u < 8; ++u) s[u] = split_scale_of(O, srow, kb + u * 32, ts);
 #pragma unroll
             for (int u = 0; u < 8; ++u) smax = max(smax, __float_as_uint(s[u]));
         }
-        for (; kb < nkb; kb += TPR) smax = max(smax, __float_as_uint(split_scale_of(O, srow, kb, ts)));
+        for (; kb < nkb; kb += 32) smax = max(smax, __float_as_uint(split_scale_of(O, srow, kb, ts)));
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) smax = max(smax, __shfl_xor_sync(0xFFFFFFFFu, smax, o));
-    if (kWarpsPerRow > 1) {
-        if (lane == 0) s_max[warp] = smax;
-        __syncthreads();
-        const int w0 = warp / kWarpsPerRow * kWarpsPerRow;
-#pragma unroll
-        for (int w = 0; w < kWarpsPerRow; ++w) smax = max(smax, s_max[w0 + w]);
-    }
     if (!active) return;
 
     // Reference 2^(e - 11), e the exponent of the largest scale: the largest normalised scale lies in [2^11, 2^12) and
@@ -223,7 +218,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
     const uint32_t bars = base + kSpOffBars;
     const uint32_t full_bar = bars, empty_bar = bars + 8 * kSpStages;
     const uint32_t tfull_bar = bars + 16 * kSpStages, tempty_bar = tfull_bar + 8;
-    const uint32_t rb_bar = tempty_bar + 8;                 // two barriers: refB of the current / the next tile
+    const uint32_t rb_bar = tempty_bar + 8;                 // two barriers: refB written / refB read by everyone
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kSpOffBars + 16 * kSpStages + 32);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
@@ -323,8 +318,8 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
         const int et = threadIdx.x - 64;
         uint8_t *buf = smem + kSpOffEpi + (warp - 2) * kSpEpiBufBytes;
         float *refb_s = reinterpret_cast<float *>(smem + kSpOffRefB);
-        int rbuf = 0;
-        uint32_t acc_phase = 0, rb_phase[2] = {0u, 0u};
+        uint32_t acc_phase = 0, rb_written = 0, rb_read = 0;
+        bool first_tile = true;
         bool ok = true;
         for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
             const TileInfo t = tile_info<2>(P, tile, rank);
@@ -334,13 +329,19 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
             const float ra = m_own < P.M ? P.refA[m_own] : 0.0f;
             {
                 const int64_t n = n0 + et;
-                refb_s[rbuf * kTN + et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
-                mbar_arrive(rb_bar + 8 * rbuf);
-                if (!mbar_wait(rb_bar + 8 * rbuf, rb_phase[rbuf], abort_flag)) { ok = false; break; }
-                rb_phase[rbuf] ^= 1u;
+                // one buffer: wait until every epilogue thread has finished with the previous tile's values, write this
+                // tile's, and wait until all of them are there (bounded, abortable waits instead of bar.sync)
+                if (!first_tile) {
+                    if (!mbar_wait(rb_bar + 8, rb_read, abort_flag)) { ok = false; break; }
+                    rb_read ^= 1u;
+                }
+                first_tile = false;
+                refb_s[et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
+                mbar_arrive(rb_bar);
+                if (!mbar_wait(rb_bar, rb_written, abort_flag)) { ok = false; break; }
+                rb_written ^= 1u;
             }
-            const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s + rbuf * kTN);
-            rbuf ^= 1;
+            const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s);
             if (has_k) {
                 if (!mbar_wait(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -374,7 +375,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                     if (m_own < t.row_end) {
                         for (int j = 0; j < 32 && n_base + j < P.N; ++j) {
                             const float sum = __fmaf_rn(__uint_as_float(v1[j]), 1.0f / kSpLoScale, __uint_as_float(v0[j]));
-                            const float val = sum * ra * refb_s[(rbuf ^ 1) * kTN + c * 32 + j];
+                            const float val = sum * ra * refb_s[c * 32 + j];
                             const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
                             if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(val);
                             else static_cast<float *>(P.C)[idx] = val;
@@ -422,6 +423,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
+            mbar_arrive(rb_bar + 8);                           // this thread has finished with the tile's refB values
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all C boxes written
         __syncwarp();

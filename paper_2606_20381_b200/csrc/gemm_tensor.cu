@@ -29,7 +29,7 @@ constexpr int kTcThreads = 64 + 32 * kEpiWarps;      // warp 0: TMA, warp 1: MMA
 constexpr int kBarrierBytes = 256;
 constexpr int kEpiBufBytes = 32 * 128;              // one staged 32-row x 32-column chunk (FP32; BF16 uses half of it)
 constexpr int kEpiBytes = kEpiWarps * kEpiBufBytes;  // one staging buffer per epilogue warp
-constexpr int kRefBBytes = 2 * kTN * 4;             // refB of the current and the next tile
+constexpr int kRefBBytes = kTN * 4;                 // refB of the current tile
 // CG = 1: one CTA per 128 x 256 tile, 4 stages of (A 128 x 128 + B 256 x 128) bytes.
 // CG = 2: a pair of CTAs (cta_group::2) per 256 x 256 tile; each CTA stages its 128 rows of A and its 128-row half of
 //         B, 6 stages of 32 KB: a third less shared-memory fill per MMA cycle, which is what bounds the main loop.
@@ -79,8 +79,7 @@ constexpr int kDecodeThreads = 256;
 // spread over more threads so that the grid has many more warps than the GPU has slots (no idle tail).
 template <int TPR>
 __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const DecodeParams P) {
-    __shared__ int s_emax[kDecodeThreads / 32];
-    constexpr int kRowsPerCta = kDecodeThreads / TPR, kWarpsPerRow = TPR / 32;
+    constexpr int kRowsPerCta = kDecodeThreads / TPR;
     if ((int64_t)blockIdx.x == P.tbl_cta) {
         if (threadIdx.x == 0) {
             int n = 0;
@@ -91,36 +90,32 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
     }
     const bool is_b = (int64_t)blockIdx.x >= P.a_ctas;
     const DecodeOperand &O = P.op[is_b ? 1 : 0];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
     const int t = threadIdx.x % TPR;
     const int64_t row = ((int64_t)blockIdx.x - (is_b ? P.a_ctas : 0)) * kRowsPerCta + threadIdx.x / TPR;
     const bool active = row < O.rows;
     const int nkb = (int)(P.K >> 4);
     const float *sptr = O.scales + (active ? row : 0) * O.lds + t;
 
-    // largest block exponent field of the row (power-of-two scales: the exponent field is the scale; 0 = zero block)
+    // largest block exponent field of the row (power-of-two scales: the exponent field is the scale; 0 = zero block).
+    // Every warp of a row scans the whole row's scales (a 32nd of the traffic; the repeats hit in cache): no shared
+    // memory and no CTA barrier, so that this kernel's CTAs fit beside a resident product-kernel CTA on the same SM.
     uint32_t fmax = 0u;
     if (active) {
         // eight loads in flight per thread: the row's scales are the first touch of DRAM, and a warp issues in order
-        int kb = t;
-        for (; kb + 7 * TPR < nkb; kb += 8 * TPR) {
+        const float *srow0 = sptr - t;
+        int kb = lane;
+        for (; kb + 7 * 32 < nkb; kb += 8 * 32) {
             uint32_t b[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) b[u] = __float_as_uint(__ldg(sptr + (kb - t) + u * TPR));
+            for (int u = 0; u < 8; ++u) b[u] = __float_as_uint(__ldg(srow0 + kb + u * 32));
 #pragma unroll
             for (int u = 0; u < 8; ++u) fmax = max(fmax, b[u]);
         }
-        for (; kb < nkb; kb += TPR) fmax = max(fmax, __float_as_uint(__ldg(sptr + (kb - t))));
+        for (; kb < nkb; kb += 32) fmax = max(fmax, __float_as_uint(__ldg(srow0 + kb)));
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) fmax = max(fmax, __shfl_xor_sync(0xFFFFFFFFu, fmax, o));
-    if (kWarpsPerRow > 1) {
-        if (lane == 0) s_emax[warp] = (int)fmax;
-        __syncthreads();
-        const int w0 = warp / kWarpsPerRow * kWarpsPerRow;      // first warp of this row
-#pragma unroll
-        for (int w = 0; w < kWarpsPerRow; ++w) fmax = max(fmax, (uint32_t)s_emax[w0 + w]);
-    }
     if (!active) return;
     // biased exponent field of the row's reference 2^eref, eref = emax - kDMax (an all-zero row takes eref = 0)
     const int fref = fmax == 0u ? 127 : (int)(fmax >> 23) - kDMax;
@@ -290,24 +285,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int et = threadIdx.x - 64;                   // 0..255 among the epilogue threads
         uint8_t *buf = smem + kOffEpi + (warp - 2) * kEpiBufBytes;
         float *refb_s = reinterpret_cast<float *>(smem + kOffRefB);
-        int acc = 0, rbuf = 0;
-        uint32_t acc_phase = 0, rb_phase[2] = {0u, 0u};
+        int acc = 0;
+        uint32_t acc_phase = 0, rb_written = 0, rb_read = 0;
+        bool first_tile = true;
         bool ok = true;
         for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
             const TileInfo t = tile_info<CG>(P, tile, rank);
             const int64_t m_own = t.m0 + q * 32 + lane;
             const float ra = m_own < P.M ? P.refA[m_own] : 0.0f;
-            // refB of this tile's 256 columns into shared memory (one value per thread), double-buffered across tiles
+            // refB of this tile's 256 columns into shared memory (one value per thread)
             {
                 const int64_t n = t.n0 + et;
-                refb_s[rbuf * kTN + et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
-                // all epilogue threads have written their value (bounded, abortable wait instead of bar.sync)
-                mbar_arrive(rb_bar + 8 * rbuf);
-                if (!mbar_wait(rb_bar + 8 * rbuf, rb_phase[rbuf], abort_flag)) { ok = false; break; }
-                rb_phase[rbuf] ^= 1u;
+                // one buffer: wait until every epilogue thread has finished with the previous tile's values, write this
+                // tile's, and wait until all of them are there (bounded, abortable waits instead of bar.sync)
+                if (!first_tile) {
+                    if (!mbar_wait(rb_bar + 8, rb_read, abort_flag)) { ok = false; break; }
+                    rb_read ^= 1u;
+                }
+                first_tile = false;
+                refb_s[et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
+                mbar_arrive(rb_bar);
+                if (!mbar_wait(rb_bar, rb_written, abort_flag)) { ok = false; break; }
+                rb_written ^= 1u;
             }
-            const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s + rbuf * kTN);
-            rbuf ^= 1;
+            const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s);
             if (t.nkb > 0) {
                 if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -343,7 +344,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // is written with plain predicated stores so that nothing right of column N is touched.
                     if (m_own < t.row_end) {
                         for (int j = 0; j < 32 && n_base + j < P.N; ++j) {
-                            const float val = __uint_as_float(v[cur][j]) * ra * refb_s[(rbuf ^ 1) * kTN + c * 32 + j];
+                            const float val = __uint_as_float(v[cur][j]) * ra * refb_s[c * 32 + j];
                             const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
                             if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(val);
                             else static_cast<float *>(P.C)[idx] = val;
@@ -388,6 +389,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
+            mbar_arrive(rb_bar + 8);                           // this thread has finished with the tile's refB values
             if (t.nkb > 0) {
                 acc ^= 1;
                 if (acc == 0) acc_phase ^= 1u;
