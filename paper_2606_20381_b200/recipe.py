@@ -12,7 +12,80 @@ import torch
 from . import binding as ufp4
 
 
-class Ufp4Linear:
+class _Ufp4Step:
+    """The schedule shared by the dense and the MoE-grouped layer: six calls, in sequence on one stream or ordered
+    only by their data dependences on three.  Subclasses provide the buffers and the calls `_quantize_x/_w/_g` and
+    `_gemm(which, workspace, stream)`."""
+
+    overlap = False
+
+    def _init_schedule(self, need_bytes: int, device, overlap: bool):
+        self.workspace = torch.empty(max(need_bytes, 16), dtype=torch.uint8, device=device)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+        # overlap: the three products run on three streams (each with its own workspace), so that the operand
+        # preparation of one product and the tails of the quantizer launches fill SMs another kernel leaves idle
+        self.overlap = overlap
+        if overlap:
+            self.workspaces = [self.workspace] + [torch.empty_like(self.workspace) for _ in range(2)]
+            self.side = [torch.cuda.Stream(device=device) for _ in range(2)]
+            self.ev = {k: torch.cuda.Event() for k in ("start", "x", "w", "g", "dx", "dw")}
+
+    def _qkw(self, stream):
+        return dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
+                    seed_rht=self.seed_rht, dev_status=self.dev_status, stream=stream)
+
+    def quantize(self, X, W, dY, stream=None):
+        self._quantize_x(X, stream)
+        self._quantize_w(W, stream)
+        self._quantize_g(dY, stream)
+
+    def gemms(self, stream=None):
+        for which in ("fwd_y", "bwd_dx", "bwd_dw"):
+            self._gemm(which, self.workspace, stream)
+
+    def step(self, X, W, dY, stream=None, join: bool = True):
+        if self.overlap:
+            return self.step_overlapped(X, W, dY, stream, join)
+        self.quantize(X, W, dY, stream)
+        self.gemms(stream)
+        return self.Y, self.dX, self.dW
+
+    def step_overlapped(self, X, W, dY, stream=None, join: bool = True):
+        """The same six calls as step(), ordered only by their data dependences: X, W and fwd_y on the caller's stream,
+        dY and bwd_dx on a second, bwd_dw on a third; the caller's stream joins both at the end (join=False leaves
+        that to a later join() call, so that independent layers overlap too)."""
+        s0 = torch.cuda.current_stream() if stream is None else stream
+        s1, s2 = self.side
+        ev = self.ev
+        ev["start"].record(s0)
+        s1.wait_event(ev["start"])
+        self._quantize_g(dY, s1)
+        ev["g"].record(s1)
+        self._quantize_x(X, s0)
+        ev["x"].record(s0)
+        self._quantize_w(W, s0)
+        ev["w"].record(s0)
+        self._gemm("fwd_y", self.workspaces[0], s0)
+        s1.wait_event(ev["w"])
+        self._gemm("bwd_dx", self.workspaces[1], s1)
+        ev["dx"].record(s1)
+        s2.wait_event(ev["g"])
+        s2.wait_event(ev["x"])
+        self._gemm("bwd_dw", self.workspaces[2], s2)
+        ev["dw"].record(s2)
+        if join:
+            self.join(s0)
+        return self.Y, self.dX, self.dW
+
+    def join(self, stream=None):
+        """Make the caller's stream wait for the side streams of the last step_overlapped()."""
+        if self.overlap:
+            s0 = torch.cuda.current_stream() if stream is None else stream
+            s0.wait_event(self.ev["dx"])
+            s0.wait_event(self.ev["dw"])
+
+
+class Ufp4Linear(_Ufp4Step):
     """Preallocated buffers and the 3-quantize + 3-GEMM step for one dense layer (T tokens, K in, N out)."""
 
     def __init__(self, tokens: int, in_features: int, out_features: int, device="cuda", grid: int = ufp4.GRID_INT4,
@@ -32,75 +105,21 @@ class Ufp4Linear:
         self.dW = torch.empty(N, K, dtype=dt, device=device)
         need = max(ufp4.gemm_workspace_bytes(self.Xr, self.Wr, path), ufp4.gemm_workspace_bytes(self.Gr, self.Wc, path),
                    ufp4.gemm_workspace_bytes(self.Gc, self.Xc, path))
-        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
-        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
-        # overlap: the three products run on three streams (each with its own workspace), so that the operand
-        # preparation of one product and the tails of the quantizer launches fill SMs another kernel leaves idle
-        self.overlap = overlap
-        if overlap:
-            self.workspaces = [self.workspace] + [torch.empty_like(self.workspace) for _ in range(2)]
-            self.side = [torch.cuda.Stream(device=device) for _ in range(2)]
-            self.ev = {k: torch.cuda.Event() for k in ("start", "x", "w", "g", "dx", "dw")}
+        self._init_schedule(need, device, overlap)
 
-    # number of kernel launches one call makes (for the benchmark's launch count)
-    launches_quantize = 3
+    def _quantize_x(self, X, stream):
+        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, **self._qkw(stream))
 
-    def quantize(self, X, W, dY, stream=None):
-        kw = dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
-                  seed_rht=self.seed_rht, dev_status=self.dev_status, stream=stream)
-        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, **kw)
-        ufp4.quantize(W, rounding=ufp4.ROUND_RTNE, out_row=self.Wr, out_col=self.Wc, **kw)
-        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, **kw)
+    def _quantize_w(self, W, stream):
+        ufp4.quantize(W, rounding=ufp4.ROUND_RTNE, out_row=self.Wr, out_col=self.Wc, **self._qkw(stream))
 
-    def gemms(self, stream=None):
-        kw = dict(path=self.path, workspace=self.workspace, dev_status=self.dev_status, stream=stream)
-        ufp4.gemm(self.Xr, self.Wr, out=self.Y, layout=ufp4.FWD_Y, **kw)
-        ufp4.gemm(self.Gr, self.Wc, out=self.dX, layout=ufp4.BWD_DX, **kw)
-        ufp4.gemm(self.Gc, self.Xc, out=self.dW, layout=ufp4.BWD_DW, **kw)
+    def _quantize_g(self, dY, stream):
+        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, **self._qkw(stream))
 
-    def step(self, X, W, dY, stream=None, join: bool = True):
-        if self.overlap:
-            return self.step_overlapped(X, W, dY, stream, join)
-        self.quantize(X, W, dY, stream)
-        self.gemms(stream)
-        return self.Y, self.dX, self.dW
-
-    def step_overlapped(self, X, W, dY, stream=None, join: bool = True):
-        """The same six calls as step(), ordered only by their data dependences: X, W and fwd_y on the caller's stream,
-        dY and bwd_dx on a second, bwd_dw on a third; the caller's stream joins both at the end (join=False leaves
-        that to a later join() call, so that independent layers overlap too)."""
-        s0 = torch.cuda.current_stream() if stream is None else stream
-        s1, s2 = self.side
-        ev = self.ev
-        qkw = dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
-                   seed_rht=self.seed_rht, dev_status=self.dev_status)
-        gkw = dict(path=self.path, dev_status=self.dev_status)
-        ev["start"].record(s0)
-        s1.wait_event(ev["start"])
-        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, stream=s1, **qkw)
-        ev["g"].record(s1)
-        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, stream=s0, **qkw)
-        ev["x"].record(s0)
-        ufp4.quantize(W, rounding=ufp4.ROUND_RTNE, out_row=self.Wr, out_col=self.Wc, stream=s0, **qkw)
-        ev["w"].record(s0)
-        ufp4.gemm(self.Xr, self.Wr, out=self.Y, layout=ufp4.FWD_Y, workspace=self.workspaces[0], stream=s0, **gkw)
-        s1.wait_event(ev["w"])
-        ufp4.gemm(self.Gr, self.Wc, out=self.dX, layout=ufp4.BWD_DX, workspace=self.workspaces[1], stream=s1, **gkw)
-        ev["dx"].record(s1)
-        s2.wait_event(ev["g"])
-        s2.wait_event(ev["x"])
-        ufp4.gemm(self.Gc, self.Xc, out=self.dW, layout=ufp4.BWD_DW, workspace=self.workspaces[2], stream=s2, **gkw)
-        ev["dw"].record(s2)
-        if join:
-            self.join(s0)
-        return self.Y, self.dX, self.dW
-
-    def join(self, stream=None):
-        """Make the caller's stream wait for the side streams of the last step_overlapped()."""
-        if self.overlap:
-            s0 = torch.cuda.current_stream() if stream is None else stream
-            s0.wait_event(self.ev["dx"])
-            s0.wait_event(self.ev["dw"])
+    def _gemm(self, which, workspace, stream):
+        a, b, out, layout = {"fwd_y": (self.Xr, self.Wr, self.Y, ufp4.FWD_Y), "bwd_dx": (self.Gr, self.Wc, self.dX, ufp4.BWD_DX),
+                             "bwd_dw": (self.Gc, self.Xc, self.dW, ufp4.BWD_DW)}[which]
+        ufp4.gemm(a, b, out=out, layout=layout, path=self.path, workspace=workspace, dev_status=self.dev_status, stream=stream)
 
     @property
     def flops(self) -> int:
@@ -111,12 +130,12 @@ class Ufp4Linear:
         return self.T * self.K + self.N * self.K + self.T * self.N
 
 
-class Ufp4MoE:
+class Ufp4MoE(_Ufp4Step):
     """The same step for an MoE expert layer: rows of X / dY grouped by expert (offsets), weights [E][F][H]."""
 
     def __init__(self, offsets_host: torch.Tensor, hidden: int, ffn: int, device="cuda", grid: int = ufp4.GRID_INT4,
                  scale_fmt: int = ufp4.SCALE_FP32, path: int = ufp4.PATH_AUTO, rht_block: int = 16, seed_rht: int = 1,
-                 seed_sr: int = 2, out_bf16: bool = False, counts: torch.Tensor | None = None):
+                 seed_sr: int = 2, out_bf16: bool = False, counts: torch.Tensor | None = None, overlap: bool = False):
         self.counts = counts
         self.offsets_host = offsets_host.to(torch.int64).contiguous()
         self.offsets_dev = self.offsets_host.to(device)
@@ -134,32 +153,24 @@ class Ufp4MoE:
         self.dW = torch.empty(E * F, H, dtype=dt, device=device)
         need = max(ufp4.gemm_workspace_bytes(self.Xr, self.Wr, path), ufp4.gemm_workspace_bytes(self.Gr, self.Wc, path),
                    ufp4.gemm_workspace_bytes(self.Gc, self.Xc, path))
-        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=device)
-        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+        self._init_schedule(need, device, overlap)
 
-    def quantize(self, X, W, dY, stream=None):
-        kw = dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
-                  seed_rht=self.seed_rht, dev_status=self.dev_status, stream=stream)
-        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, **kw)
-        ufp4.quantize_batched(W.view(self.E, self.F, self.H), rounding=ufp4.ROUND_RTNE, out_row=self.Wr,
-                              out_col=self.Wc, **kw)
-        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, **kw)
+    def _quantize_x(self, X, stream):
+        ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, **self._qkw(stream))
 
-    def gemms(self, stream=None):
-        kw = dict(path=self.path, workspace=self.workspace, dev_status=self.dev_status, stream=stream)
-        ufp4.gemm_grouped(self.Xr, self.Wr, self.offsets_dev, self.offsets_host, self.F, ufp4.FWD_Y, out=self.Y, **kw)
-        ufp4.gemm_grouped(self.Gr, self.Wc, self.offsets_dev, self.offsets_host, self.H, ufp4.BWD_DX, out=self.dX, **kw)
-        ufp4.gemm_grouped(self.Gc, self.Xc, self.offsets_dev, self.offsets_host, self.F, ufp4.BWD_DW, out=self.dW, **kw)
+    def _quantize_w(self, W, stream):
+        ufp4.quantize_batched(W.view(self.E, self.F, self.H), rounding=ufp4.ROUND_RTNE, out_row=self.Wr, out_col=self.Wc,
+                              **self._qkw(stream))
 
-    overlap = False     # the grouped step runs its calls in sequence on one stream
+    def _quantize_g(self, dY, stream):
+        ufp4.quantize(dY, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc, **self._qkw(stream))
 
-    def step(self, X, W, dY, stream=None, join: bool = True):
-        self.quantize(X, W, dY, stream)
-        self.gemms(stream)
-        return self.Y, self.dX, self.dW
-
-    def join(self, stream=None):
-        pass
+    def _gemm(self, which, workspace, stream):
+        a, b, out, layout, gn = {"fwd_y": (self.Xr, self.Wr, self.Y, ufp4.FWD_Y, self.F),
+                                 "bwd_dx": (self.Gr, self.Wc, self.dX, ufp4.BWD_DX, self.H),
+                                 "bwd_dw": (self.Gc, self.Xc, self.dW, ufp4.BWD_DW, self.F)}[which]
+        ufp4.gemm_grouped(a, b, self.offsets_dev, self.offsets_host, gn, layout, out=out, path=self.path, workspace=workspace,
+                          dev_status=self.dev_status, stream=stream)
 
     @property
     def flops(self) -> int:
