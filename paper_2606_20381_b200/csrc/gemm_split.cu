@@ -185,10 +185,13 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
                 lw[2 * q + h] = *reinterpret_cast<const uint32_t *>(&lo2);
             }
         }
-        hptr[2 * kb] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-        hptr[2 * kb + 1] = make_uint4(hw[4], hw[5], hw[6], hw[7]);
-        lptr[2 * kb] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-        lptr[2 * kb + 1] = make_uint4(lw[4], lw[5], lw[6], lw[7]);
+        // one 32-byte store per block and piece (rows are 32-byte aligned: K is a multiple of 16)
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     :: "l"(hptr + 2 * kb), "r"(hw[0]), "r"(hw[1]), "r"(hw[2]), "r"(hw[3]), "r"(hw[4]), "r"(hw[5]), "r"(hw[6]), "r"(hw[7])
+                     : "memory");
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     :: "l"(lptr + 2 * kb), "r"(lw[0]), "r"(lw[1]), "r"(lw[2]), "r"(lw[3]), "r"(lw[4]), "r"(lw[5]), "r"(lw[6]), "r"(lw[7])
+                     : "memory");
     }
     if (flushed != 0u && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
 }
