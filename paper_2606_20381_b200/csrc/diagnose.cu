@@ -19,6 +19,7 @@ struct DiagParams {
     const float *scales;
     int64_t ldc, lds;
     int grid, rht;
+    int load256;                   // x and its row pitch are 32-byte aligned: 256-bit loads
     uint32_t sign_mask;
     double *partials;              // [gridDim.x][kDiagSums]
 };
@@ -52,7 +53,14 @@ __global__ void __launch_bounds__(kDiagThreads) diagnose_kernel(const DiagParams
     for (int64_t blk = (int64_t)blockIdx.x * kDiagThreads + threadIdx.x; blk < nblk; blk += (int64_t)gridDim.x * kDiagThreads) {
         const int64_t r = blk / bpr, b = blk - r * bpr;
         const uint4 *src = reinterpret_cast<const uint4 *>(P.x + r * P.ld + 16 * b);
-        const uint4 d0 = __ldg(src), d1 = __ldg(src + 1);
+        uint4 d0, d1;
+        if (P.load256) {
+            asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(d0.x), "=r"(d0.y), "=r"(d0.z), "=r"(d0.w), "=r"(d1.x), "=r"(d1.y), "=r"(d1.z), "=r"(d1.w) : "l"(src));
+        } else {
+            d0 = __ldg(src);
+            d1 = __ldg(src + 1);
+        }
         const uint2 cw = __ldg(reinterpret_cast<const uint2 *>(P.codes + r * P.ldc + 8 * b));
         const float s = __ldg(P.scales + r * P.lds + b);
         const uint32_t w[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
@@ -160,6 +168,7 @@ extern "C" int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t 
     P.scales = static_cast<const float *>(q_row->scales);
     P.ldc = q_row->ld_codes_bytes; P.lds = q_row->ld_scales;
     P.grid = q_row->grid; P.rht = rht_block == 16;
+    P.load256 = ufp4::aligned_to(x, 32) && ld % 16 == 0;
     P.sign_mask = ufp4_rht_sign_mask(seed_rht);
     P.partials = static_cast<double *>(workspace);
     const int64_t nblk = rows * (cols / 16);

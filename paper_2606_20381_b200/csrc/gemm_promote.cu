@@ -100,8 +100,10 @@ __global__ void __launch_bounds__(256) decode_promote_kernel(const PDecodeParams
             }
             out[j] = pair;
         }
-        optr[2 * kb] = make_uint4(out[0], out[1], out[2], out[3]);
-        optr[2 * kb + 1] = make_uint4(out[4], out[5], out[6], out[7]);
+        // one 32-byte store per block (rows are 32-byte aligned: K is a multiple of 16)
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                     :: "l"(optr + 2 * kb), "r"(out[0]), "r"(out[1]), "r"(out[2]), "r"(out[3]), "r"(out[4]), "r"(out[5]), "r"(out[6]), "r"(out[7])
+                     : "memory");
     }
 }
 
