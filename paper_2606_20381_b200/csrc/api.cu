@@ -114,7 +114,7 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     const bool pow2 = A->scale_fmt == UFP4_SCALE_POW2 && B->scale_fmt == UFP4_SCALE_POW2;
     if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
         return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
-    // AUTO may take SPLIT (plain products) or PROMOTE (grouped products): enough for either
+    // AUTO takes SPLIT, and PROMOTE only where SPLIT does not apply: enough for either
     const size_t split = ufp4::gemm_split_workspace_bytes(A->rows, B->rows, A->k);
     const size_t promote = ufp4::gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
     if (path == UFP4_PATH_SPLIT) return split;

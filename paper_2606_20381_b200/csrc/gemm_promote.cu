@@ -1,7 +1,8 @@
 // Tensor-core path of the block-scaled 4-bit GEMM (Sec. 2.2: Y^ = Q_G(XH') Q_G(WH')^T) for arbitrary FP32 block scales
 // (Table 1's "FP32 single-level" scale, and the E4M3 x tensor two-level format).
 //
-// code x FP32 scale needs up to 27 significant bits, so it cannot be folded into any tensor-core operand.  Instead the
+// code x FP32 scale needs up to 27 significant bits, so it cannot be folded into any single tensor-core operand (the
+// split path carries it as two FP16 pieces and is the faster of the two; this path is taken on request).  Here the
 // integer codes go to the tensor cores and the scales to the CUDA cores: per 16-element quant block one
 // tcgen05.mma kind::f16 (K = 16, BF16 operands holding the exact integers q, FP32 accumulation, no carry-in) writes the
 // exact integer partial P_kb[m][n] of a 128 x 128 tile into tensor memory, and eight "promotion" warps read it back
@@ -11,7 +12,7 @@
 //   1. decode_promote_kernel: packed nibbles -> BF16 integers [rows][K]; scales -> FP32, transposed to [K/16][rows] so that
 //      a stage's scales land in shared memory as contiguous per-block rows (caller's workspace).
 //   2. gemm_promote_kernel: persistent; warp 0 TMA producer (4-stage ring: A, B, sA, sB), warp 1 MMA issuer (one MMA per
-//      quant block into two alternating 128-column tensor-memory buffers), warps 2-9 promotion + epilogue (TMA stores).
+//      quant block into four alternating 128-column tensor-memory buffers), warps 2-9 promotion + epilogue (TMA stores).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
