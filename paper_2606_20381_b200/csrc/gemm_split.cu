@@ -211,7 +211,8 @@ __device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t adesc,
 
 // One pair of CTAs per 256 x 256 tile of C; the CTA of rank r holds rows [m0 + 128 r, +128) of both A pieces and rows
 // [n0 + 128 r, +128) of both B pieces.  Accumulator 0 (columns 0..255 of tensor memory) takes hi_a hi_b, accumulator 1
-// (columns 256..511) takes hi_a lo_b + lo_a hi_b.
+// (columns 256..511) takes hi_a lo_b + lo_a hi_b.  Tiles, reduction ranges and expert rows come from tile_info: plain
+// products, row-grouped products (256-row tiles laid out group by group) and reduction-grouped products alike.
 __global__ void __launch_bounds__(kSpThreads, 1)
 gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
                   const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl,
