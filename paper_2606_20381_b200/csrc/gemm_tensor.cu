@@ -96,6 +96,19 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
     const bool active = row < O.rows;
     const int nkb = (int)(P.K >> 4);
     const float *sptr = O.scales + (active ? row : 0) * O.lds + t;
+    const uint2 *cptr = reinterpret_cast<const uint2 *>(O.codes + (active ? row : 0) * O.ldc) + t;
+
+    // the thread's first kPre blocks (codes and exponent fields) are requested before the scan below, so that their
+    // trip to DRAM overlaps the scan's
+    constexpr int kPre = 4;
+    uint2 pcw[kPre];
+    int pf[kPre];
+#pragma unroll
+    for (int u = 0; u < kPre; ++u) {
+        const bool in = active && t + u * TPR < nkb;
+        pcw[u] = in ? __ldg(cptr + u * TPR) : make_uint2(0u, 0u);
+        pf[u] = in ? (int)(__float_as_uint(__ldg(sptr + u * TPR)) >> 23) : 0;   // scales are non-negative: no sign bit
+    }
 
     // largest block exponent field of the row (power-of-two scales: the exponent field is the scale; 0 = zero block).
     // Every warp of a row scans the whole row's scales (a 32nd of the traffic; the repeats hit in cache): no shared
@@ -138,12 +151,8 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
     const uint32_t mul_nlo = int4 ? 0x04040404u : 0x04040400u;     // a zero entry stays zero
     const int fkeep = max(1, fref + kDMin);                        // smallest exponent field that is not flushed
     uint32_t flushed = 0u;
-    const uint2 *cptr = reinterpret_cast<const uint2 *>(O.codes + row * O.ldc) + t;
     uint4 *optr = reinterpret_cast<uint4 *>(O.out8 + row * P.K) + t;
-#pragma unroll 4
-    for (int kb = t; kb < nkb; kb += TPR, cptr += TPR, optr += TPR, sptr += TPR) {
-        const int f = (int)(__float_as_uint(__ldg(sptr)) >> 23);   // scales are non-negative: no sign bit to mask
-        uint2 cw = __ldg(cptr);
+    auto emit = [&](int f, uint2 cw, uint4 *dst) {
         // a zero-scale or flushed block decodes as all-zero codes (table entry 0 is 0 at every d)
         const bool keep = f >= fkeep;
         flushed |= (keep || f == 0) ? 0u : (cw.x | cw.y);
@@ -164,8 +173,15 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
             const uint32_t pos = __byte_perm(lutp_lo, lutp_hi, sel), neg = __byte_perm(lutn_lo, lutn_hi, sel);
             out[q] = __byte_perm(pos, neg, ((w >> 1) & 0x4444u) | 0x3210u);
         }
-        *optr = make_uint4(out[0], out[1], out[2], out[3]);
-    }
+        *dst = make_uint4(out[0], out[1], out[2], out[3]);
+    };
+#pragma unroll
+    for (int u = 0; u < kPre; ++u)
+        if (t + u * TPR < nkb) emit(pf[u], pcw[u], optr + u * TPR);
+    cptr += kPre * TPR; optr += kPre * TPR; sptr += kPre * TPR;
+#pragma unroll 4
+    for (int kb = t + kPre * TPR; kb < nkb; kb += TPR, cptr += TPR, optr += TPR, sptr += TPR)
+        emit((int)(__float_as_uint(__ldg(sptr)) >> 23), __ldg(cptr), optr);
     if (flushed != 0u && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
 }
 
