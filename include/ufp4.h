@@ -159,6 +159,7 @@ size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, i
  *          only); blocks whose exponent lies outside a row's window set UFP4_DEV_EXP_WINDOW.
  * PROMOTE: tcgen05 computes the exact integer partial of every 16-element block (BF16 operands, K = 16 per MMA) and the
  *          CUDA cores promote it with sA * sB into FP32 accumulators; every grid and scale format (Table 1's FP32 scales).
+ *          A row-grouped product needs group_n % 4 == 0 on this path (else UFP4_ERR_UNSUPPORTED; AUTO moves on to EXACT).
  * SPLIT:   tcgen05 / TMEM kernel on FP16 operands: each dequantized value, relative to a per-row power-of-two
  *          reference, is split into two FP16 pieces (22 significant bits) and the product taken by three MMAs per K
  *          step; every grid and scale format (Table 1's FP32 scales), plain and grouped; blocks more than 2^26 below

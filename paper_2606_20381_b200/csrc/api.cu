@@ -19,6 +19,7 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
 
 size_t gemm_promote_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
 int gemm_promote_kernel_launches();
+bool gemm_promote_supported(int mode, int64_t group_n);
 int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                         int64_t M, int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n,
                         void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
@@ -71,7 +72,9 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
         if (path == UFP4_PATH_SPLIT) return UFP4_ERR_WORKSPACE;
     }
     // PROMOTE, or AUTO for what neither tensor-core operand form can take
-    {
+    const bool promote_ok = gemm_promote_supported(mode, group_n);
+    if (path == UFP4_PATH_PROMOTE && !promote_ok) return UFP4_ERR_UNSUPPORTED;
+    if (promote_ok) {
         const size_t need = gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
         if (workspace && workspace_bytes >= need)
             return gemm_promote_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, workspace,

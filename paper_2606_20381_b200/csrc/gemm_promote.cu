@@ -379,6 +379,10 @@ size_t gemm_promote_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K) {
 
 int gemm_promote_kernel_launches() { return 2; }
 
+// The transposed scales of B are fetched by TMA starting at column b_row0 + n0 (FP32): in a row-grouped product
+// b_row0 = group * group_n, which must stay 16-byte aligned.
+bool gemm_promote_supported(int mode, int64_t group_n) { return mode != 1 || group_n % 4 == 0; }
+
 static bool pmake_map(CUtensorMap *map, CUtensorMapDataType dt, const void *ptr, uint64_t inner, uint64_t outer,
                       uint64_t stride_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle sw) {
     EncodeTiledFn fn = encode_tiled_fn();
@@ -394,6 +398,7 @@ static bool pmake_map(CUtensorMap *map, CUtensorMapDataType dt, const void *ptr,
 int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                         int64_t M, int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n,
                         void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
+    if (!gemm_promote_supported(mode, group_n)) return UFP4_ERR_UNSUPPORTED;
     if (!aligned_to(workspace, 256)) return UFP4_ERR_ALIGN;
     if (workspace_bytes < gemm_promote_workspace_bytes(A->rows, B->rows, K)) return UFP4_ERR_WORKSPACE;
     if (A->rows > 0x7FFFFFFF || B->rows > 0x7FFFFFFF || K > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
