@@ -17,6 +17,7 @@ import numpy as np
 from .build import build as _build
 
 GRID_INT4, GRID_E1M2, GRID_E2M1 = 0, 1, 2
+GRID_E2M1_MAX4, GRID_E2M1_MAX2 = 3, 4      # E2M1 with the magnitudes above 4 / above 2 unused (Sec. 5.4, max_fpx)
 ROUND_RTNE, ROUND_SR = 0, 1
 SCALE_FP32, SCALE_POW2, SCALE_E4M3_TENSOR = 0, 1, 2
 AXIS_ROW, AXIS_COL = 0, 1
@@ -33,6 +34,8 @@ def lib():
         L.orc_level.argtypes = [i32, i32]
         L.orc_gmax.restype = f64
         L.orc_gmax.argtypes = [i32]
+        L.orc_num_levels.restype = i32
+        L.orc_num_levels.argtypes = [i32]
         L.orc_philox4x32_10.restype = None
         L.orc_philox4x32_10.argtypes = [p, p, p]
         L.orc_rht_sign_mask.restype = C.c_uint32

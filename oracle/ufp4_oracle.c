@@ -31,6 +31,8 @@
  *     key = seed; the 16 little-endian bytes of the four output words are the elements' random bytes r;
  *     round up iff p * 256 > r + 0.5, p being the exact fractional position between the two neighbouring levels.
  *   - A block with amax == 0 or amax < 2^-100 is stored as scale 0, codes 0.  Zero is always nibble 0x0.
+ *   - Range-restricted E2M1 (Sec. 5.4, `max_fpx` of App. B): g_max = max_fpx in the scale, and rho_G rounds onto the
+ *     E2M1 levels not above max_fpx (max_fpx = 2 keeps {0, 0.5, 1, 1.5, 2}); encoding and dequantization are E2M1's.
  *
  * Parity pins: see tests/test_oracle_pins.py.  The E4M3-with-tensor-scale mode has no counterpart in the paper and
  * is pinned only by brute force: "parity unpinned" by the paper for that mode.
@@ -42,7 +44,9 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORC_GRID_INT4 = 0, ORC_GRID_E1M2 = 1, ORC_GRID_E2M1 = 2 };
+/* E2M1_MAX4 / E2M1_MAX2: the E2M1 codebook with the magnitudes above 4 / above 2 left unused (the range-restricted
+ * E2M1 of Sec. 5.4 and App. B's `max_fpx`): g_max = 4 / 2, same nibble encoding as E2M1. */
+enum { ORC_GRID_INT4 = 0, ORC_GRID_E1M2 = 1, ORC_GRID_E2M1 = 2, ORC_GRID_E2M1_MAX4 = 3, ORC_GRID_E2M1_MAX2 = 4 };
 enum { ORC_ROUND_RTNE = 0, ORC_ROUND_SR = 1 };
 enum { ORC_SCALE_FP32 = 0, ORC_SCALE_POW2 = 1, ORC_SCALE_E4M3_TENSOR = 2 };
 enum { ORC_AXIS_ROW = 0, ORC_AXIS_COL = 1 };
@@ -61,10 +65,13 @@ static const double *levels_of(int grid) {
     }
 }
 
-/* Non-negative level i (0..7) of a grid; exported so tests can read the codebook. */
+/* Number of non-negative levels in use: a range-restricted grid keeps the levels up to its g_max. */
+int orc_num_levels(int grid) { return grid == ORC_GRID_E2M1_MAX4 ? 7 : (grid == ORC_GRID_E2M1_MAX2 ? 5 : 8); }
+
+/* Non-negative level i (0..7) of a grid's codebook; exported so tests can read the codebook. */
 double orc_level(int grid, int i) { return levels_of(grid)[i & 7]; }
 
-double orc_gmax(int grid) { return levels_of(grid)[7]; }
+double orc_gmax(int grid) { return levels_of(grid)[orc_num_levels(grid) - 1]; }
 
 /* ---------------------------------------------------------------- Philox4x32-10 (Salmon et al., SC'11) */
 
@@ -142,9 +149,10 @@ void orc_rht16_f32(float v[16], uint32_t sign_mask) {
  * values above the top level saturate to it. */
 int orc_round_rtne(double a, int grid) {
     const double *L = levels_of(grid);
+    const int n = orc_num_levels(grid);
     int best = 0;
     double best_d = fabs(a - L[0]);
-    for (int i = 1; i < 8; ++i) {
+    for (int i = 1; i < n; ++i) {
         double d = fabs(a - L[i]);
         if (d < best_d || (d == best_d && (i % 2 == 0))) {
             best = i;
@@ -158,9 +166,10 @@ int orc_round_rtne(double a, int grid) {
  * taken iff p * 256 > r + 0.5, p = (a - g_a) / (g_b - g_a); at or above the top level the top level is taken. */
 int orc_round_sr(double a, int grid, int r) {
     const double *L = levels_of(grid);
-    if (a >= L[7]) return 7;
+    const int n = orc_num_levels(grid);
+    if (a >= L[n - 1]) return n - 1;
     int lo = 0;
-    for (int i = 1; i < 8; ++i)
+    for (int i = 1; i < n; ++i)
         if (L[i] <= a) lo = i;
     double p = (a - L[lo]) / (L[lo + 1] - L[lo]);
     return (p * 256.0 > (double)r + 0.5) ? lo + 1 : lo;
@@ -296,7 +305,7 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int 
                  uint8_t *codes, void *scales, float *y_out) {
     if (!x || !codes || !scales) return -1;
     if (rht_block != 0 && rht_block != 16) return -1;
-    if (grid < 0 || grid > 2 || rounding < 0 || rounding > 1 || scale_fmt < 0 || scale_fmt > 2) return -1;
+    if (grid < 0 || grid > 4 || rounding < 0 || rounding > 1 || scale_fmt < 0 || scale_fmt > 2) return -1;
     int64_t R = (axis == ORC_AXIS_ROW) ? rows : cols; /* output rows   */
     int64_t K = (axis == ORC_AXIS_ROW) ? cols : rows; /* reduction dim */
     if (K % 16 != 0 || R <= 0 || K <= 0) return -1;

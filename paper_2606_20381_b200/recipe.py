@@ -34,23 +34,26 @@ class _Ufp4Step:
         return dict(axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt,
                     seed_rht=self.seed_rht, dev_status=self.dev_status, stream=stream)
 
-    def quantize(self, X, W, dY, stream=None):
+    def quantize(self, X, W, dY, stream=None, reuse_w: bool = False):
         self._quantize_x(X, stream)
-        self._quantize_w(W, stream)
+        if not reuse_w:
+            self._quantize_w(W, stream)
         self._quantize_g(dY, stream)
 
     def gemms(self, stream=None):
         for which in ("fwd_y", "bwd_dx", "bwd_dw"):
             self._gemm(which, self.workspace, stream)
 
-    def step(self, X, W, dY, stream=None, join: bool = True):
+    def step(self, X, W, dY, stream=None, join: bool = True, reuse_w: bool = False):
+        """reuse_w: W has not changed since the last step (micro-batches of one optimizer step): its two quantized
+        variants are kept and only X and dY are quantized (RTNE of the same W gives the same codes)."""
         if self.overlap:
-            return self.step_overlapped(X, W, dY, stream, join)
-        self.quantize(X, W, dY, stream)
+            return self.step_overlapped(X, W, dY, stream, join, reuse_w)
+        self.quantize(X, W, dY, stream, reuse_w)
         self.gemms(stream)
         return self.Y, self.dX, self.dW
 
-    def step_overlapped(self, X, W, dY, stream=None, join: bool = True):
+    def step_overlapped(self, X, W, dY, stream=None, join: bool = True, reuse_w: bool = False):
         """The same six calls as step(), ordered only by their data dependences: X, W and fwd_y on the caller's stream,
         dY and bwd_dx on a second, bwd_dw on a third; the caller's stream joins both at the end (join=False leaves
         that to a later join() call, so that independent layers overlap too)."""
@@ -63,7 +66,8 @@ class _Ufp4Step:
         ev["g"].record(s1)
         self._quantize_x(X, s0)
         ev["x"].record(s0)
-        self._quantize_w(W, s0)
+        if not reuse_w:
+            self._quantize_w(W, s0)
         ev["w"].record(s0)
         self._gemm("fwd_y", self.workspaces[0], s0)
         s1.wait_event(ev["w"])

@@ -11,7 +11,7 @@ import pytest
 import torch
 
 import oracle
-from oracle import (AXIS_COL, AXIS_ROW, GRID_E1M2, GRID_E2M1, GRID_INT4, ROUND_RTNE, ROUND_SR, SCALE_E4M3_TENSOR,
+from oracle import (AXIS_COL, AXIS_ROW, GRID_E1M2, GRID_E2M1, GRID_E2M1_MAX2, GRID_E2M1_MAX4, GRID_INT4, ROUND_RTNE, ROUND_SR, SCALE_E4M3_TENSOR,
                     SCALE_FP32, SCALE_POW2)
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -149,7 +149,7 @@ def test_nibble_encodings():
 def _exact_rtne(a: Fraction, levels):
     """Nearest level in exact rational arithmetic; ties to the even index."""
     best, best_d = 0, abs(a - levels[0])
-    for i in range(1, 8):
+    for i in range(1, len(levels)):
         d = abs(a - levels[i])
         if d < best_d or (d == best_d and i % 2 == 0):
             best, best_d = i, d
@@ -312,6 +312,63 @@ def test_scale_is_amax_over_gmax_and_top_code_is_used(grid, gmax):
     lo, hi = q.codes & 0xF, q.codes >> 4
     vals = np.vectorize(lambda n: abs(oracle.nibble_value(grid, int(n))))(np.stack([lo, hi], -1).reshape(48, 4, 16))
     assert np.all(vals.max(axis=2) == gmax)          # no clipping and s = amax / g_max: the top level is always hit
+
+
+# ------------------------------------------------------------------ range-restricted E2M1 (Sec. 5.4; App. B, max_fpx)
+
+@pytest.mark.parametrize("grid,max_fpx,kept", [(GRID_E2M1_MAX4, 4.0, [0, 0.5, 1, 1.5, 2, 3, 4]),
+                                               (GRID_E2M1_MAX2, 2.0, [0, 0.5, 1, 1.5, 2])])
+def test_range_restricted_e2m1_levels_scale_and_rounding(grid, max_fpx, kept):
+    """Sec. 5.4: max_fpx = 2 keeps only {0, 0.5, 1, 1.5, 2}; the scale divides by max_fpx, the codes are E2M1 codes,
+    nothing above max_fpx is ever emitted and the block maximum lands on max_fpx."""
+    assert oracle.lib().orc_gmax(grid) == max_fpx
+    assert list(oracle.levels(grid)) == list(oracle.levels(GRID_E2M1))          # same codebook behind the nibbles
+    for n in range(16):
+        assert oracle.nibble_value(grid, n) == oracle.nibble_value(GRID_E2M1, n)
+    # rounding onto the kept levels only: brute force over a fine sweep, exact rational nearest-level search
+    Lf = [Fraction(v) for v in kept]
+    for a in np.linspace(0.0, 7.0, 1401):
+        assert oracle.levels(grid)[oracle.round_rtne(float(a), grid)] == float(Lf[_exact_rtne(Fraction(float(a)), Lf)])
+        out = {oracle.levels(grid)[oracle.round_sr(float(a), grid, r)] for r in (0, 100, 255)}
+        lo = max(v for v in kept if v <= min(a, max_fpx))
+        hi = min([v for v in kept if v > a] + [max_fpx])
+        assert out <= {lo, hi}
+    # through the quantizer
+    bits = _rand_bits(48, 64, 31, 0.37)
+    amax = np.abs(bf16_vals(bits)).reshape(48, 4, 16).max(axis=2)
+    for rounding in (ROUND_RTNE, ROUND_SR):
+        q = oracle.quantize(bits, AXIS_ROW, rht_block=0, grid=grid, rounding=rounding, seed_sr=4)
+        assert np.array_equal(q.scales, (amax.astype(np.float32) / np.float32(max_fpx)).astype(np.float32))
+        mags = np.abs(oracle.dequantize(q) / np.repeat(q.scales.astype(np.float64), 16, axis=1))
+        assert set(np.unique(mags).tolist()) <= set(kept)
+        assert np.all(mags.reshape(48, 4, 16).max(axis=2) == max_fpx)
+
+
+def test_max_fpx_2_is_a_uniform_five_level_grid():
+    """With max_fpx = 2 the kept levels are the integers 0..4 in half units: the quantizer must agree with a plain
+    uniform quantizer, round-half-even of 2 x / s clipped to 4 (numpy's rint), in value and in E2M1 nibble."""
+    bits = _rand_bits(40, 96, 32, 2.5)
+    x = bf16_vals(bits).astype(np.float32)
+    q = oracle.quantize(bits, AXIS_ROW, rht_block=0, grid=GRID_E2M1_MAX2)
+    amax = np.abs(x).reshape(40, 6, 16).max(axis=2)
+    inv = (np.float32(2.0) / amax.astype(np.float32)).astype(np.float32)
+    y = (x * np.repeat(inv, 16, axis=1)).astype(np.float32)
+    k = np.clip(np.rint(2.0 * np.abs(y.astype(np.float64))), 0, 4).astype(np.int64)      # level index = half units
+    nib = np.where((y < 0) & (k > 0), 8 | k, k).astype(np.uint8)
+    assert np.array_equal(q.codes, nib[:, 0::2] | (nib[:, 1::2] << 4))
+
+
+def test_max_fpx_6_is_the_unrestricted_e2m1():
+    """max_fpx = 6 is the E2M1 reference itself (App. B): the restricted rounding rule with all eight levels kept."""
+    L = oracle.levels(GRID_E2M1)
+    assert oracle.lib().orc_gmax(GRID_E2M1) == 6.0 and oracle.lib().orc_num_levels(GRID_E2M1) == 8
+    assert oracle.lib().orc_num_levels(GRID_E2M1_MAX4) == 7 and oracle.lib().orc_num_levels(GRID_E2M1_MAX2) == 5
+    for a in np.linspace(0, 4.0, 161):          # below the first dropped midpoint all three rules agree ...
+        if a < 1.99:
+            assert oracle.round_rtne(float(a), GRID_E2M1) == oracle.round_rtne(float(a), GRID_E2M1_MAX2)
+        if a < 3.99:
+            assert oracle.round_rtne(float(a), GRID_E2M1) == oracle.round_rtne(float(a), GRID_E2M1_MAX4)
+    assert L[oracle.round_rtne(5.5, GRID_E2M1)] == 6.0 and L[oracle.round_rtne(5.5, GRID_E2M1_MAX4)] == 4.0
 
 
 def test_e1m2_is_int4_with_scale_times_four():
