@@ -48,8 +48,13 @@ typedef enum {
 /* Data-element grids (Sec. 2.1; Sec. 3.1 prints the E2M1 magnitudes).  INT4 and E1M2 are the same uniform grid:
  * INT4 stores q in [-7,7] as a two's-complement nibble with g_max = 7; E1M2 stores sign|e|mm with values q/4 and
  * g_max = 1.75, so its block scale is exactly 4x the INT4 one.  E2M1 is the comparison grid {0,.5,1,1.5,2,3,4,6}
- * stored as sign|ee|m.  Zero is always encoded as nibble 0x0. */
-typedef enum { UFP4_GRID_INT4 = 0, UFP4_GRID_E1M2 = 1, UFP4_GRID_E2M1 = 2 } ufp4_grid;
+ * stored as sign|ee|m.  Zero is always encoded as nibble 0x0.
+ * E2M1_MAX4 / E2M1_MAX2 are the range-restricted E2M1 of Sec. 5.4 (App. B's `max_fpx` = 4 / 2): the quantizer scales by
+ * g_max = 4 / 2 and rounds onto the E2M1 levels not above it (max_fpx = 2 keeps {0,.5,1,1.5,2}); the codes are E2M1
+ * codes, so the GEMM and diagnostics calls read such a tensor exactly like an E2M1 one. */
+typedef enum {
+    UFP4_GRID_INT4 = 0, UFP4_GRID_E1M2 = 1, UFP4_GRID_E2M1 = 2, UFP4_GRID_E2M1_MAX4 = 3, UFP4_GRID_E2M1_MAX2 = 4
+} ufp4_grid;
 
 /* Rounding rule rho_G (Sec. 2.1).  RTNE: nearest level, ties to the even code.  SR: between neighbouring levels
  * g_a <= t < g_b the upper one is taken with probability (t - g_a)/(g_b - g_a), resolved to 1/256 by one random byte

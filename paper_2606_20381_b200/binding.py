@@ -12,6 +12,7 @@ from dataclasses import dataclass
 import torch
 
 GRID_INT4, GRID_E1M2, GRID_E2M1 = 0, 1, 2
+GRID_E2M1_MAX4, GRID_E2M1_MAX2 = 3, 4      # range-restricted E2M1 (Sec. 5.4, max_fpx = 4 / 2): quantizer-side only
 ROUND_RTNE, ROUND_SR = 0, 1
 AXIS_ROW, AXIS_COL, AXIS_BOTH = 0, 1, 2
 SCALE_FP32, SCALE_POW2, SCALE_E4M3_TENSOR = 0, 1, 2

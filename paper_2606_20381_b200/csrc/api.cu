@@ -33,7 +33,7 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
 
 static int check_operand(const ufp4_qtensor *q) {
     if (!q || !q->codes || !q->scales) return UFP4_ERR_NULL;
-    if (q->grid < 0 || q->grid > 2 || q->scale_fmt < 0 || q->scale_fmt > 2) return UFP4_ERR_ENUM;
+    if (q->grid < 0 || q->grid > 4 || q->scale_fmt < 0 || q->scale_fmt > 2) return UFP4_ERR_ENUM;
     if (q->rows < 1 || q->k < 16 || q->k % 16 != 0) return UFP4_ERR_SHAPE;
     if (q->ld_codes_bytes < q->k / 2 || q->ld_codes_bytes % 16 != 0 || q->ld_scales < q->k / 16) return UFP4_ERR_ALIGN;
     if (!aligned_to(q->codes, 16)) return UFP4_ERR_ALIGN;

@@ -36,6 +36,9 @@ __host__ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t 
 constexpr uint32_t kRhtCounterTag = 0x52485400u;  // counter word 3 of the sign draw
 constexpr uint32_t kSrCounterTag = 0x53520000u;   // counter word 3 of the SR draws
 
+// The codebook behind a tensor's nibbles: the range-restricted E2M1 grids store plain E2M1 codes.
+inline int codebook_of(int grid) { return grid > UFP4_GRID_E2M1 ? (int)UFP4_GRID_E2M1 : grid; }
+
 inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 #define UFP4_CUDA_OK(expr)                                \

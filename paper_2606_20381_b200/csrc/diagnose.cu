@@ -155,7 +155,7 @@ extern "C" int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t 
     if (!x || !q_row || !q_row->codes || !q_row->scales || !dev_out || !workspace) return UFP4_ERR_NULL;
     if (rows < 1 || cols < 16 || cols % 16 != 0 || ld < cols || q_row->rows != rows || q_row->k != cols) return UFP4_ERR_SHAPE;
     if (rht_block != 0 && rht_block != 16) return UFP4_ERR_UNSUPPORTED;
-    if (q_row->grid < 0 || q_row->grid > 2) return UFP4_ERR_ENUM;
+    if (q_row->grid < 0 || q_row->grid > 4) return UFP4_ERR_ENUM;
     if (q_row->scale_fmt == UFP4_SCALE_E4M3_TENSOR) return UFP4_ERR_UNSUPPORTED;
     if (!ufp4::aligned_to(x, 16) || (ld * 2) % 16 != 0 || !ufp4::aligned_to(q_row->codes, 8) || q_row->ld_codes_bytes % 8 != 0 ||
         !ufp4::aligned_to(dev_out, 8) || !ufp4::aligned_to(workspace, 8))
@@ -167,7 +167,7 @@ extern "C" int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t 
     P.codes = static_cast<const uint8_t *>(q_row->codes);
     P.scales = static_cast<const float *>(q_row->scales);
     P.ldc = q_row->ld_codes_bytes; P.lds = q_row->ld_scales;
-    P.grid = q_row->grid; P.rht = rht_block == 16;
+    P.grid = ufp4::codebook_of(q_row->grid); P.rht = rht_block == 16;
     P.load256 = ufp4::aligned_to(x, 32) && ld % 16 == 0;
     P.sign_mask = ufp4_rht_sign_mask(seed_rht);
     P.partials = static_cast<double *>(workspace);

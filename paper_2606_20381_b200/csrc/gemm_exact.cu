@@ -176,9 +176,9 @@ int gemm_exact_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
                       void *stream) {
     ExactParams P = {};
     P.A = OperandView{static_cast<const uint8_t *>(A->codes), A->scales, A->tensor_scale, A->ld_codes_bytes, A->ld_scales,
-                      A->grid, A->scale_fmt};
+                      codebook_of(A->grid), A->scale_fmt};
     P.B = OperandView{static_cast<const uint8_t *>(B->codes), B->scales, B->tensor_scale, B->ld_codes_bytes, B->ld_scales,
-                      B->grid, B->scale_fmt};
+                      codebook_of(B->grid), B->scale_fmt};
     P.C = C; P.ldc = ldc; P.c_is_bf16 = c_is_bf16;
     P.M = M; P.N = N; P.K = K; P.mode = mode;
     P.offsets = offsets; P.num_groups = num_groups; P.group_n = group_n;

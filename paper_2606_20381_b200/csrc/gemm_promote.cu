@@ -412,9 +412,9 @@ int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, i
 
     PDecodeParams D = {};
     D.op[0] = PDecodeOperand{static_cast<const uint8_t *>(A->codes), A->scales, A->tensor_scale, A->ld_codes_bytes,
-                             A->ld_scales, A->rows, lda_t, A->grid, A->scale_fmt, A16, sAt};
+                             A->ld_scales, A->rows, lda_t, codebook_of(A->grid), A->scale_fmt, A16, sAt};
     D.op[1] = PDecodeOperand{static_cast<const uint8_t *>(B->codes), B->scales, B->tensor_scale, B->ld_codes_bytes,
-                             B->ld_scales, B->rows, ldb_t, B->grid, B->scale_fmt, B16, sBt};
+                             B->ld_scales, B->rows, ldb_t, codebook_of(B->grid), B->scale_fmt, B16, sBt};
     D.K = K;
     D.a_ctas = (A->rows + 7) / 8;
     const int64_t decode_ctas = D.a_ctas + (B->rows + 7) / 8;

@@ -503,9 +503,9 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
 
     SDecodeParams D = {};
     D.op[0] = SDecodeOperand{static_cast<const uint8_t *>(A->codes), A->scales, A->tensor_scale, A->ld_codes_bytes,
-                             A->ld_scales, A->rows, A->grid, A->scale_fmt, Ah, Al, refA};
+                             A->ld_scales, A->rows, codebook_of(A->grid), A->scale_fmt, Ah, Al, refA};
     D.op[1] = SDecodeOperand{static_cast<const uint8_t *>(B->codes), B->scales, B->tensor_scale, B->ld_codes_bytes,
-                             B->ld_scales, B->rows, B->grid, B->scale_fmt, Bh, Bl, refB};
+                             B->ld_scales, B->rows, codebook_of(B->grid), B->scale_fmt, Bh, Bl, refB};
     D.K = K;
     D.dev_status = dev_status;
     int tpr = 32;           // a warp per row up to 8 blocks per thread, more threads on longer rows

@@ -490,9 +490,9 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
 
     DecodeParams D = {};
     D.op[0] = DecodeOperand{static_cast<const uint8_t *>(A->codes), static_cast<const float *>(A->scales),
-                            A->ld_codes_bytes, A->ld_scales, A->rows, A->grid, A8, refA};
+                            A->ld_codes_bytes, A->ld_scales, A->rows, codebook_of(A->grid), A8, refA};
     D.op[1] = DecodeOperand{static_cast<const uint8_t *>(B->codes), static_cast<const float *>(B->scales),
-                            B->ld_codes_bytes, B->ld_scales, B->rows, B->grid, B8, refB};
+                            B->ld_codes_bytes, B->ld_scales, B->rows, codebook_of(B->grid), B8, refB};
     D.K = K;
     int tpr = 32;           // a warp per row up to 8 blocks per thread, more threads on longer rows
     while (tpr < kDecodeThreads && (K >> 4) >= (int64_t)16 * tpr) tpr *= 2;

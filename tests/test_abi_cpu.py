@@ -75,7 +75,7 @@ def test_quantize_rejects_bad_arguments_without_launching(lib):
     assert call(x=None) == -1
     assert call(row=None) == -1
     assert call(col=None) == -1
-    assert call(axis=5) == -4 and call(grid=3) == -4 and call(rnd=2) == -4 and call(fmt=9) == -4
+    assert call(axis=5) == -4 and call(grid=5) == -4 and call(rnd=2) == -4 and call(fmt=9) == -4
     assert call(rht=32) == -5
     assert call(cols=40, ld=40) == -2                    # cols % 16
     assert call(rows=40) == -2                           # rows % 16 for the col variant

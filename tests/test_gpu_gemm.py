@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from helpers import assert_gemm_close, oracle_quantize, to_device
+from helpers import assert_gemm_close, assert_qtensor_equal, oracle_quantize, to_device
 from paper_2606_20381_b200 import binding as ufp4
 from paper_2606_20381_b200 import inputs
 
@@ -173,3 +173,26 @@ def test_split_path_exponent_window_and_extreme_scales():
     A = oracle_quantize(torch.from_numpy(x).bfloat16(), oracle.AXIS_ROW, **kw)
     ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_SPLIT, dev_status=status)
     assert int(status.item()) & ufp4.DEV_EXP_WINDOW
+
+
+@pytest.mark.parametrize("grid", [ufp4.GRID_E2M1_MAX4, ufp4.GRID_E2M1_MAX2])
+def test_range_restricted_e2m1_operands_on_every_path(grid):
+    """Sec. 5.4's range-restricted E2M1 (max_fpx = 4 / 2): quantized on the GPU, bit-equal to the oracle, and read by
+    every GEMM path as the E2M1 codes they are."""
+    M, N, K = 200, 136, 320
+    X = inputs.heavy_tailed_activations(M, K, seed=61)
+    W = inputs.normal_bf16(N, K, 0.02, seed=62)
+    for scale_fmt, paths in ((oracle.SCALE_POW2, (ufp4.PATH_TENSOR, ufp4.PATH_SPLIT, ufp4.PATH_EXACT)),
+                             (oracle.SCALE_FP32, (ufp4.PATH_SPLIT, ufp4.PATH_PROMOTE, ufp4.PATH_EXACT, ufp4.PATH_AUTO))):
+        kw = dict(rht_block=16, grid=grid, scale_fmt=scale_fmt, seed_rht=1)
+        A, _ = ufp4.quantize(X.cuda(), axis=ufp4.AXIS_ROW, **kw)
+        B, _ = ufp4.quantize(W.cuda(), axis=ufp4.AXIS_ROW, **kw)
+        Ao, Bo = oracle_quantize(X, oracle.AXIS_ROW, **kw), oracle_quantize(W, oracle.AXIS_ROW, **kw)
+        assert_qtensor_equal(A, Ao, "A")
+        assert_qtensor_equal(B, Bo, "B")
+        ref, S = oracle.gemm(Ao, Bo)
+        for path in paths:
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            out = ufp4.gemm(A, B, path=path, dev_status=status)
+            assert int(status.item()) == 0
+            assert_gemm_close(out.cpu().numpy(), ref, S, f"grid {grid} fmt {scale_fmt} path {path}")

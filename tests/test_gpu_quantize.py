@@ -10,7 +10,7 @@ from paper_2606_20381_b200 import inputs
 
 pytestmark = pytest.mark.gpu
 
-GRIDS = [ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1]
+GRIDS = [ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1, ufp4.GRID_E2M1_MAX4, ufp4.GRID_E2M1_MAX2]
 
 
 def run_both(x, axis, **kw):
@@ -47,7 +47,8 @@ def test_all_variants_on_a_ragged_multi_tile_matrix(grid, rounding, scale_fmt, r
     x = inputs.spiky_normal(272, 400, seed=5)          # 3 x 4 tiles of 128 with ragged edges in both directions
     kw = dict(rht_block=rht_block, grid=grid, rounding=rounding, scale_fmt=scale_fmt, seed_rht=3, seed_sr=11)
     if scale_fmt == ufp4.SCALE_E4M3_TENSOR:
-        gmax = {ufp4.GRID_INT4: 7.0, ufp4.GRID_E1M2: 1.75, ufp4.GRID_E2M1: 6.0}[grid]
+        gmax = {ufp4.GRID_INT4: 7.0, ufp4.GRID_E1M2: 1.75, ufp4.GRID_E2M1: 6.0, ufp4.GRID_E2M1_MAX4: 4.0,
+                ufp4.GRID_E2M1_MAX2: 2.0}[grid]
         kw["tensor_scale"] = float(np.float32(4.0 * x.float().abs().max().item() / (gmax * 448.0)))
     run_both(x, ufp4.AXIS_BOTH, **kw)
 
@@ -161,7 +162,7 @@ def test_tensor_diagnostics_agree_with_the_oracle():
     from paper_2606_20381_b200 import diagnostics
     x = inputs.spiky_normal(520, 1040, seed=3)
     xb = inputs.bf16_bits(x)
-    for grid in (ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1):
+    for grid in GRIDS:
         for rht in (0, 16):
             row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=rht, grid=grid, seed_rht=1)
             got = diagnostics.tensor_diagnostics(x.cuda(), row, rht, 1)
@@ -185,6 +186,12 @@ def test_tensor_diagnostics_agree_with_the_oracle():
     row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_INT4, seed_rht=1)
     _, b = diagnostics.per_bin_bias(x.cuda(), row, 16, 1)
     assert abs(b[1:7]).max() < 0.05     # what remains is the decreasing density inside symmetric bins, not geometry
+    # Sec. 5.4: restricting E2M1 to magnitudes <= 2 removes the asymmetric bins but gives up bucket utilization
+    row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_E2M1_MAX2, seed_rht=1)
+    d2 = diagnostics.tensor_diagnostics(x.cuda(), row, 16, 1)
+    assert d2["count"][5:].sum() == 0 and abs(d2["bias"][1:4]).max() < 0.05
+    row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_E2M1, seed_rht=1)
+    assert d2["b_eff"] < diagnostics.tensor_diagnostics(x.cuda(), row, 16, 1)["b_eff"]
 
 
 def test_rht_helps_the_uniform_grid_more_than_e2m1_on_outlier_heavy_tensors():

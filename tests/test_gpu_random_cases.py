@@ -20,7 +20,8 @@ def _bf16(a):
 @pytest.mark.parametrize("seed", [0, 1, 2, 3])
 def test_quantizer_random_cases(seed):
     """Ten cases per seed: R, C in 16..624; plain normal, per-row scaling over 2^+-110 (subnormal and near-overflow
-    blocks), per-element scaling over 2^+-30, 70 % zeros, quarter-integer values (exact rounding ties)."""
+    blocks), per-element scaling over 2^+-30, 70 % zeros, quarter-integer values (exact rounding ties); all five grids
+    (the range-restricted E2M1 variants included)."""
     rng = np.random.default_rng(1000 + seed)
     for _ in range(10):
         R, C = 16 * int(rng.integers(1, 40)), 16 * int(rng.integers(1, 40))
@@ -35,7 +36,7 @@ def test_quantizer_random_cases(seed):
         elif mode == 4:
             x = np.round(x * 4) / 4 * np.exp2(rng.integers(-5, 5))
         xt = _bf16(x)
-        kw = dict(rht_block=16 * int(rng.integers(0, 2)), grid=int(rng.integers(0, 3)), rounding=int(rng.integers(0, 2)),
+        kw = dict(rht_block=16 * int(rng.integers(0, 2)), grid=int(rng.integers(0, 5)), rounding=int(rng.integers(0, 2)),
                   scale_fmt=int(rng.integers(0, 2)), seed_rht=int(rng.integers(0, 1 << 40)), seed_sr=int(rng.integers(0, 1 << 40)))
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         row, col = ufp4.quantize(xt.cuda(), axis=ufp4.AXIS_BOTH, dev_status=status, **kw)
