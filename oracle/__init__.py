@@ -44,6 +44,10 @@ def lib():
         L.orc_sr_bytes.argtypes = [u64, u64, C.c_uint32, p]
         L.orc_hadamard_matrix.restype = None
         L.orc_hadamard_matrix.argtypes = [i32, p]
+        L.orc_rht_signs.restype = None
+        L.orc_rht_signs.argtypes = [u64, p]
+        L.orc_rht_f32.restype = None
+        L.orc_rht_f32.argtypes = [p, i32, p]
         L.orc_rht16_f32.restype = None
         L.orc_rht16_f32.argtypes = [p, C.c_uint32]
         L.orc_round_rtne.restype = i32
@@ -129,6 +133,21 @@ def rht16_f32(v, sign_mask: int) -> np.ndarray:
     a = np.ascontiguousarray(v, dtype=np.float32).copy()
     assert a.shape == (16,)
     lib().orc_rht16_f32(_ptr(a), sign_mask)
+    return a
+
+
+def rht_signs(seed: int) -> np.ndarray:
+    """The 128 sign bits of a seed as four 32-bit words (bit i set: eps_i = -1)."""
+    out = np.zeros(4, dtype=np.uint32)
+    lib().orc_rht_signs(seed, _ptr(out))
+    return out
+
+
+def rht_f32(v, n: int, signs: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(v, dtype=np.float32).copy()
+    assert a.shape == (n,) and n in (32, 64, 128)
+    s = np.ascontiguousarray(signs, dtype=np.uint32)
+    lib().orc_rht_f32(_ptr(a), n, _ptr(s))
     return a
 
 

@@ -8,6 +8,7 @@
  * What each function follows:
  *   orc_hadamard_matrix   Sec. 2.2, the Sylvester recursion H_2n = 1/sqrt(2) [[H,H],[H,-H]], H_1 = [1]
  *   orc_rht16_f32         Sec. 2.2, H'_16 = S_16 H_16 applied to a row vector (signs first, then Hadamard), FP32
+ *   orc_rht_f32           the same for the RHT block sizes 32 / 64 / 128 of App. B's search space
  *   orc_quantize          Sec. 2.1, s_B = max|x_j| / g_max, q_i = rho_G(x_i / s_B); Sec. 4 / Table 1 (1x16 blocks,
  *                         FP32 single-level scale, RHT block 16); Sec. 2.2 last paragraph (blocks and RHT run along
  *                         the reduction dimension, so a tensor has a "row" and a "col" variant)
@@ -101,6 +102,14 @@ uint32_t orc_rht_sign_mask(uint64_t seed) {
     return out[0] & 0xFFFFu;
 }
 
+/* The sign bits of RHT blocks up to 128 wide: bit i of the 128-bit output of the same Philox call (word i / 32,
+ * bit i % 32) set means eps_i = -1; the 16-point mask above is its first 16 bits. */
+void orc_rht_signs(uint64_t seed, uint32_t out[4]) {
+    uint32_t ctr[4] = {0, 0, 0, 0x52485400u};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    orc_philox4x32_10(ctr, key, out);
+}
+
 /* The 16 random bytes of quant block b of a variant (0 = row, 1 = col). */
 void orc_sr_bytes(uint64_t seed_sr, uint64_t block_index, uint32_t variant, uint8_t r[16]) {
     uint32_t ctr[4] = {(uint32_t)block_index, (uint32_t)(block_index >> 32), variant, 0x53520000u};
@@ -141,6 +150,23 @@ void orc_rht16_f32(float v[16], uint32_t sign_mask) {
                 v[i + h] = a - b;
             }
     for (int i = 0; i < 16; ++i) v[i] = 0.25f * v[i];
+}
+
+/* v <- (v o eps) H_n in FP32 for n = 32, 64, 128 (App. B lists these block sizes beside the selected 16): signs, the
+ * butterfly stages h = 1, 2, ..., n/2 in that order, then one multiplication by the FP32 value nearest to 1/sqrt(n)
+ * (exact for n = 64). */
+void orc_rht_f32(float *v, int n, const uint32_t signs[4]) {
+    for (int i = 0; i < n; ++i)
+        if ((signs[i >> 5] >> (i & 31)) & 1u) v[i] = -v[i];
+    for (int h = 1; h < n; h *= 2)
+        for (int i = 0; i < n; ++i)
+            if ((i & h) == 0) {
+                float a = v[i], b = v[i + h];
+                v[i] = a + b;
+                v[i + h] = a - b;
+            }
+    const float c = (float)(1.0 / sqrt((double)n));
+    for (int i = 0; i < n; ++i) v[i] = c * v[i];
 }
 
 /* ---------------------------------------------------------------- rounding rules (Sec. 2.1) */
@@ -304,19 +330,39 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int 
                  int rounding, int scale_fmt, uint64_t seed_rht, uint64_t seed_sr, float tensor_scale,
                  uint8_t *codes, void *scales, float *y_out) {
     if (!x || !codes || !scales) return -1;
-    if (rht_block != 0 && rht_block != 16) return -1;
+    if (rht_block != 0 && rht_block != 16 && rht_block != 32 && rht_block != 64 && rht_block != 128) return -1;
     if (grid < 0 || grid > 4 || rounding < 0 || rounding > 1 || scale_fmt < 0 || scale_fmt > 2) return -1;
     int64_t R = (axis == ORC_AXIS_ROW) ? rows : cols; /* output rows   */
     int64_t K = (axis == ORC_AXIS_ROW) ? cols : rows; /* reduction dim */
     if (K % 16 != 0 || R <= 0 || K <= 0) return -1;
+    if (rht_block > 16 && K % rht_block != 0) return -1;
 
-    orc_params p = {grid, rounding, scale_fmt, rht_block, orc_rht_sign_mask(seed_rht), seed_sr, tensor_scale};
+    /* RHT blocks wider than the quant block: the whole rht_block-wide chunk is rotated first, then its 16-element
+     * blocks are quantized without further rotation. */
+    const int wide = rht_block > 16;
+    uint32_t signs[4];
+    orc_rht_signs(seed_rht, signs);
+    orc_params p = {grid, rounding, scale_fmt, wide ? 0 : rht_block, orc_rht_sign_mask(seed_rht), seed_sr, tensor_scale};
     int64_t nkb = K / 16;
+    float chunk[128];
     for (int64_t o = 0; o < R; ++o)
         for (int64_t kb = 0; kb < nkb; ++kb) {
             float xb[16];
+            if (wide && (kb * 16) % rht_block == 0) {
+                for (int i = 0; i < rht_block; ++i) {
+                    int64_t k = kb * 16 + i;
+                    uint16_t h = (axis == ORC_AXIS_ROW) ? x[o * ld + k] : x[k * ld + o];
+                    uint32_t u = (uint32_t)h << 16;
+                    memcpy(&chunk[i], &u, 4);
+                }
+                orc_rht_f32(chunk, rht_block, signs);
+            }
             for (int i = 0; i < 16; ++i) {
                 int64_t k = kb * 16 + i;
+                if (wide) {
+                    xb[i] = chunk[k % rht_block];
+                    continue;
+                }
                 uint16_t h = (axis == ORC_AXIS_ROW) ? x[o * ld + k] : x[k * ld + o];
                 uint32_t u = (uint32_t)h << 16;
                 memcpy(&xb[i], &u, 4);

@@ -100,6 +100,61 @@ def test_rht_is_invertible_and_preserves_the_gemm():
     assert np.allclose(back, x, atol=1e-6)
 
 
+@pytest.mark.parametrize("n", [32, 64, 128])
+def test_wide_rht_equals_row_vector_times_sign_times_hadamard(n):
+    """RHT block sizes 32 / 64 / 128 (App. B): v -> (v o eps) H_n with the Sylvester H_n, signs first; the 128 sign bits
+    are the four Philox words whose first 16 bits are the 16-point mask."""
+    H = oracle.hadamard_matrix(n)
+    c32 = float(np.float32(1.0 / np.sqrt(n)))
+    for seed in (0, 1, 0xDEADBEEFCAFEF00D):
+        signs = oracle.rht_signs(seed)
+        w = oracle.philox4x32_10([0, 0, 0, 0x52485400], [seed & 0xFFFFFFFF, seed >> 32])
+        assert np.array_equal(signs, w) and int(signs[0]) & 0xFFFF == oracle.rht_sign_mask(seed)
+        eps = np.array([-1.0 if (int(signs[i >> 5]) >> (i & 31)) & 1 else 1.0 for i in range(n)])
+        Hp = np.diag(eps) @ H
+        assert np.max(np.abs(Hp @ Hp.T - np.eye(n))) < 1e-15
+        for i in (0, 1, 15, 16, 17, n // 2, n - 1):              # basis vectors: row i of H', up to the FP32 1/sqrt(n)
+            e = np.zeros(n, dtype=np.float32)
+            e[i] = 1.0
+            assert np.array_equal(oracle.rht_f32(e, n, signs).astype(np.float64), np.sign(Hp[i]) * c32)
+        rng = np.random.default_rng(seed & 0xFFFF)
+        x = rng.integers(-64, 64, size=n).astype(np.float32)     # small integers: every butterfly step is exact
+        want = (x.astype(np.float64) @ (np.sign(Hp))).astype(np.float32) * np.float32(c32)
+        assert np.array_equal(oracle.rht_f32(x, n, signs), want.astype(np.float32))
+        x = rng.standard_normal(n).astype(np.float32)
+        assert np.allclose(oracle.rht_f32(x, n, signs), x.astype(np.float64) @ Hp, rtol=0, atol=4e-6)
+
+
+@pytest.mark.parametrize("n", [32, 64, 128])
+def test_wide_rht_quantizer_rotates_whole_chunks_then_quantizes_16_blocks(n):
+    """Quantizing with RHT block n equals quantizing, without rotation, the tensor whose n-wide chunks along the
+    reduction dimension were rotated beforehand (values that stay BF16-exact: small integers times a power of two, so
+    that the pre-rotated tensor can be handed over in BF16), for both layouts; and the rotation preserves the product."""
+    rng = np.random.default_rng(n)
+    signs = oracle.rht_signs(5)
+    rows, cols = 2 * n, 2 * n
+    # entries in {-1, 0, 1} times 2^k: chunk sums stay below 2^8 in magnitude, exact in BF16 after the power-of-two part
+    x = rng.integers(-1, 2, size=(rows, cols)).astype(np.float32)
+    bits = bf16_bits(x)
+    for axis in (AXIS_ROW, AXIS_COL):
+        xs = x if axis == AXIS_ROW else x.T
+        rot = np.stack([np.concatenate([oracle.rht_f32(r[c:c + n], n, signs) for c in range(0, r.size, n)]) for r in xs])
+        if n == 64:                                   # 1/8 is exact: the rotated tensor is itself BF16-exact
+            assert np.array_equal(bf16_vals(bf16_bits(rot)), rot.astype(np.float64))
+            pre = bf16_bits(rot if axis == AXIS_ROW else rot.T)
+            a = oracle.quantize(bits, axis, rht_block=n, seed_rht=5)
+            b = oracle.quantize(pre, axis, rht_block=0)
+            assert np.array_equal(a.codes, b.codes) and np.array_equal(a.scales, b.scales)
+        # any n: the scale of every block is amax of the rotated values over g_max
+        q = oracle.quantize(bits, axis, rht_block=n, seed_rht=5)
+        amax = np.abs(rot).reshape(rot.shape[0], -1, 16).max(axis=2).astype(np.float32)
+        assert np.array_equal(q.scales, (amax / np.float32(7.0)).astype(np.float32))
+    # the rotation is orthogonal up to the rounding of 1/sqrt(n): products of rotated operands match the plain product
+    X, W = rng.standard_normal((8, 2 * n)).astype(np.float32), rng.standard_normal((6, 2 * n)).astype(np.float32)
+    rot = lambda M: np.stack([np.concatenate([oracle.rht_f32(r[c:c + n], n, signs) for c in range(0, r.size, n)]) for r in M])
+    assert np.allclose(rot(X).astype(np.float64) @ rot(W).astype(np.float64).T, X.astype(np.float64) @ W.astype(np.float64).T, atol=2e-5)
+
+
 def test_sign_mask_depends_on_seed_only_through_philox_word0():
     for seed in (0, 1, 2, 0xDEADBEEFCAFEF00D):
         w = oracle.philox4x32_10([0, 0, 0, 0x52485400], [seed & 0xFFFFFFFF, seed >> 32])
