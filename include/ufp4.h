@@ -107,6 +107,11 @@ const char *ufp4_status_string(int status);
  * Bits are the low 16 bits of word 0 of Philox4x32-10 with counter (0,0,0,0x52485400) and key (lo32, hi32) of seed. */
 uint32_t ufp4_rht_sign_mask(uint64_t seed_rht);
 
+/* The sign bits of the wider RHT blocks (32 / 64 / 128, the sizes App. B lists beside the selected 16): all 128 bits of
+ * the same Philox output, bit i (word i / 32, bit i % 32) set meaning eps_i = -1; the mask above is its first 16 bits.
+ * Host computation; out is host memory. */
+void ufp4_rht_signs(uint64_t seed_rht, uint32_t out[4]);
+
 /* Densely packed sizes of a [rows][k] quantized tensor (ld_codes_bytes = k/2 rounded up to 16, ld_scales = k/16). */
 int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t *codes_bytes, size_t *scales_bytes);
 
@@ -118,7 +123,10 @@ int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t *codes_byt
  *   axis       ROW needs cols % 16 == 0 and fills *out_row = [rows][cols];
  *              COL needs rows % 16 == 0 and cols % 16 == 0 and fills *out_col = [cols][rows];
  *              BOTH fills both from a single read of x
- *   rht_block  0 (no rotation) or 16
+ *   rht_block  0 (no rotation), 16 (the recipe's choice, Table 1), or 32 / 64 / 128 (App. B's other candidates: the
+ *              reduction dimension of each requested variant must then be a multiple of rht_block; the rotated values
+ *              are scaled by RN(1 / sqrt(rht_block)) in FP32 and their 16-element blocks quantized as usual; a plain,
+ *              slower kernel)
  *   seed_rht   selects the sign vector (ufp4_rht_sign_mask); along COL the sign of row r is eps_(r mod 16)
  *   seed_sr    key of the SR random bytes; counter = (lo32(b), hi32(b), variant, 0x53520000), b = index of the block in
  *              the variant's dense [rows][k/16] scale array, variant 0 = row, 1 = col

@@ -32,6 +32,9 @@
  *     key = seed; the 16 little-endian bytes of the four output words are the elements' random bytes r;
  *     round up iff p * 256 > r + 0.5, p being the exact fractional position between the two neighbouring levels.
  *   - A block with amax == 0 or amax < 2^-100 is stored as scale 0, codes 0.  Zero is always nibble 0x0.
+ *   - RHT blocks of 32 / 64 / 128 (App. B): sign i of the block is bit i of all 128 bits of that Philox output;
+ *     butterfly stages h = 1, 2, ..., n/2 in FP32, then one multiplication by the FP32 value nearest 1/sqrt(n); the
+ *     quant blocks stay 16 wide and are taken from the rotated chunk.
  *   - Range-restricted E2M1 (Sec. 5.4, `max_fpx` of App. B): g_max = max_fpx in the scale, and rho_G rounds onto the
  *     E2M1 levels not above max_fpx (max_fpx = 2 keeps {0, 0.5, 1, 1.5, 2}); encoding and dequantization are E2M1's.
  *

@@ -23,7 +23,7 @@ DEV_NONFINITE, DEV_EXP_WINDOW, DEV_WAIT_TIMEOUT = 1, 2, 4
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libufp4.so")
 
-EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_qtensor_bytes", "ufp4_quantize",
+EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_rht_signs", "ufp4_qtensor_bytes", "ufp4_quantize",
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
            "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes"]
 
@@ -53,6 +53,8 @@ def lib():
         L.ufp4_status_string.argtypes = [i32]
         L.ufp4_rht_sign_mask.restype = C.c_uint32
         L.ufp4_rht_sign_mask.argtypes = [u64]
+        L.ufp4_rht_signs.restype = None
+        L.ufp4_rht_signs.argtypes = [u64, C.POINTER(C.c_uint32)]
         L.ufp4_qtensor_bytes.restype = i32
         L.ufp4_qtensor_bytes.argtypes = [i64, i64, i32, C.POINTER(sz), C.POINTER(sz)]
         L.ufp4_quantize.restype = i32
@@ -126,6 +128,13 @@ class QTensor:
 
 def rht_sign_mask(seed: int) -> int:
     return int(lib().ufp4_rht_sign_mask(seed))
+
+
+def rht_signs(seed: int) -> list:
+    """The 128 sign bits of the wider RHT blocks as four 32-bit words."""
+    out = (C.c_uint32 * 4)()
+    lib().ufp4_rht_signs(seed, out)
+    return [int(v) for v in out]
 
 
 def alloc_qtensor(rows: int, k: int, grid: int, scale_fmt: int, device, tensor_scale=None) -> QTensor:

@@ -46,6 +46,12 @@ def test_sign_mask_matches_oracle(lib):
         assert ufp4.rht_sign_mask(seed) == oracle.rht_sign_mask(seed)
 
 
+def test_wide_rht_signs_match_oracle(lib):
+    for seed in (0, 1, 2, 12345, 0xDEADBEEFCAFEF00D):
+        got = ufp4.rht_signs(seed)
+        assert got == [int(v) for v in oracle.rht_signs(seed)] and got[0] & 0xFFFF == ufp4.rht_sign_mask(seed)
+
+
 def test_qtensor_bytes(lib):
     cb, sb = C.c_size_t(), C.c_size_t()
     assert lib.ufp4_qtensor_bytes(100, 48, 0, C.byref(cb), C.byref(sb)) == 0
@@ -76,7 +82,7 @@ def test_quantize_rejects_bad_arguments_without_launching(lib):
     assert call(row=None) == -1
     assert call(col=None) == -1
     assert call(axis=5) == -4 and call(grid=5) == -4 and call(rnd=2) == -4 and call(fmt=9) == -4
-    assert call(rht=32) == -5
+    assert call(rht=48) == -5 and call(rht=128) == -2   # unknown block size; reduction dimensions not multiples of 128
     assert call(cols=40, ld=40) == -2                    # cols % 16
     assert call(rows=40) == -2                           # rows % 16 for the col variant
     assert call(x=x + 2) == -3 and call(ld=68) == -3     # 16-byte alignment of x and its rows

@@ -53,6 +53,48 @@ def test_all_variants_on_a_ragged_multi_tile_matrix(grid, rounding, scale_fmt, r
     run_both(x, ufp4.AXIS_BOTH, **kw)
 
 
+@pytest.mark.parametrize("rht_block,shape", [(32, (288, 160)), (64, (320, 192)), (128, (384, 256)), (128, (128, 128))])
+@pytest.mark.parametrize("grid", [ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1])
+@pytest.mark.parametrize("rounding", [ufp4.ROUND_RTNE, ufp4.ROUND_SR])
+@pytest.mark.parametrize("scale_fmt", [ufp4.SCALE_FP32, ufp4.SCALE_POW2, ufp4.SCALE_E4M3_TENSOR])
+def test_wide_rht_blocks(rht_block, shape, grid, rounding, scale_fmt):
+    """RHT blocks of 32 / 64 / 128 (the block sizes App. B lists beside the selected 16) on multi-tile matrices with
+    ragged tile edges: both layouts bit-equal to the oracle."""
+    x = inputs.spiky_normal(shape[0], shape[1], seed=rht_block + shape[0])
+    kw = dict(rht_block=rht_block, grid=grid, rounding=rounding, scale_fmt=scale_fmt, seed_rht=7, seed_sr=13)
+    if scale_fmt == ufp4.SCALE_E4M3_TENSOR:
+        gmax = {ufp4.GRID_INT4: 7.0, ufp4.GRID_E1M2: 1.75, ufp4.GRID_E2M1: 6.0}[grid]
+        kw["tensor_scale"] = float(np.float32(4.0 * x.float().abs().max().item() / (gmax * 448.0)))
+    run_both(x, ufp4.AXIS_BOTH, **kw)
+
+
+def test_wide_rht_single_axis_and_shape_rules():
+    x = inputs.normal_bf16(48, 256, 1.0, seed=3)            # 48 rows: the row variant alone takes any row count
+    run_both(x, ufp4.AXIS_ROW, rht_block=128, seed_rht=2)
+    x = inputs.normal_bf16(192, 80, 1.0, seed=4)            # 80 columns: the col variant alone only needs rows % 64 == 0
+    run_both(x, ufp4.AXIS_COL, rht_block=64, seed_rht=2)
+    with pytest.raises(ufp4.Ufp4Error):                     # cols = 80 is not a multiple of 32
+        ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=32)
+    with pytest.raises(ufp4.Ufp4Error):
+        ufp4.quantize(x.cuda(), axis=ufp4.AXIS_BOTH, rht_block=48)
+
+
+def test_wide_rht_operands_feed_the_gemm():
+    """Rotating both operands with the same 64-wide RHT leaves the product unchanged up to quantization: the GEMM of the
+    GPU-quantized operands equals the oracle's GEMM of the oracle-quantized ones."""
+    from helpers import assert_gemm_close
+    X = inputs.heavy_tailed_activations(256, 512, seed=71)
+    W = inputs.normal_bf16(192, 512, 0.02, seed=72)
+    kw = dict(rht_block=64, scale_fmt=ufp4.SCALE_POW2, seed_rht=3)
+    A, _ = ufp4.quantize(X.cuda(), axis=ufp4.AXIS_ROW, **kw)
+    B, _ = ufp4.quantize(W.cuda(), axis=ufp4.AXIS_ROW, **kw)
+    ref, S = oracle.gemm(oracle_quantize(X, oracle.AXIS_ROW, **kw), oracle_quantize(W, oracle.AXIS_ROW, **kw))
+    out = ufp4.gemm(A, B)
+    assert_gemm_close(out.cpu().numpy(), ref, S, "rht 64")
+    plain = X.double() @ W.double().T
+    assert float((out.cpu().double() - plain).norm() / plain.norm()) < 0.2
+
+
 @pytest.mark.parametrize("shape", [(16, 16), (128, 128), (16, 2048), (2048, 16), (144, 16), (1040, 1296)])
 def test_shapes(shape):
     x = inputs.heavy_tailed_activations(shape[0], shape[1], seed=shape[0] + shape[1])
