@@ -174,6 +174,14 @@ def test_batched_weights_stack_along_rows():
         assert_qtensor_equal(col.row_slice(e * K, (e + 1) * K), ref, f"col variant of expert {e}")
     with pytest.raises(ufp4.Ufp4Error):
         ufp4.quantize_batched(W.cuda().view(E, N, K), rounding=ufp4.ROUND_SR)
+    # the same with a 64-wide RHT block (the plain kernel): 3 experts of 64 x 192
+    E, N, K = 3, 64, 192
+    W = inputs.normal_bf16(E * N, K, 0.02, seed=16)
+    row, col = ufp4.quantize_batched(W.cuda().view(E, N, K), axis=ufp4.AXIS_BOTH, rht_block=64, seed_rht=8)
+    assert_qtensor_equal(row, oracle_quantize(W, oracle.AXIS_ROW, rht_block=64, seed_rht=8), "stacked row variant, rht 64")
+    for e in range(E):
+        ref = oracle_quantize(W[e * N:(e + 1) * N], oracle.AXIS_COL, rht_block=64, seed_rht=8)
+        assert_qtensor_equal(col.row_slice(e * K, (e + 1) * K), ref, f"col variant of expert {e}, rht 64")
 
 
 def test_repeated_runs_are_bit_identical():
