@@ -20,6 +20,7 @@ GRID_INT4, GRID_E1M2, GRID_E2M1 = 0, 1, 2
 GRID_E2M1_MAX4, GRID_E2M1_MAX2 = 3, 4      # E2M1 with the magnitudes above 4 / above 2 unused (Sec. 5.4, max_fpx)
 ROUND_RTNE, ROUND_SR = 0, 1
 SCALE_FP32, SCALE_POW2, SCALE_E4M3_TENSOR = 0, 1, 2
+SCALE_E8M0_B32 = 3      # one power-of-two scale per 32 elements (MXFP4's block layout), stored per 16-element half
 AXIS_ROW, AXIS_COL = 0, 1
 
 _lib = None

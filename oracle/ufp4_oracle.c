@@ -35,6 +35,9 @@
  *   - RHT blocks of 32 / 64 / 128 (App. B): sign i of the block is bit i of all 128 bits of that Philox output;
  *     butterfly stages h = 1, 2, ..., n/2 in FP32, then one multiplication by the FP32 value nearest 1/sqrt(n); the
  *     quant blocks stay 16 wide and are taken from the rotated chunk.
+ *   - 1x32 blocks with an E8M0 scale (Sec. 2.1's footnote on MXFP4): amax over the 32 rotated elements, scale = the
+ *     next power of two >= amax / g_max (E8M0 holds exactly the powers of two), shared by the two 16-element halves;
+ *     rotation, rounding, SR draws and block indices stay per 16 elements.
  *   - Range-restricted E2M1 (Sec. 5.4, `max_fpx` of App. B): g_max = max_fpx in the scale, and rho_G rounds onto the
  *     E2M1 levels not above max_fpx (max_fpx = 2 keeps {0, 0.5, 1, 1.5, 2}); encoding and dequantization are E2M1's.
  *
@@ -52,7 +55,9 @@
  * E2M1 of Sec. 5.4 and App. B's `max_fpx`): g_max = 4 / 2, same nibble encoding as E2M1. */
 enum { ORC_GRID_INT4 = 0, ORC_GRID_E1M2 = 1, ORC_GRID_E2M1 = 2, ORC_GRID_E2M1_MAX4 = 3, ORC_GRID_E2M1_MAX2 = 4 };
 enum { ORC_ROUND_RTNE = 0, ORC_ROUND_SR = 1 };
-enum { ORC_SCALE_FP32 = 0, ORC_SCALE_POW2 = 1, ORC_SCALE_E4M3_TENSOR = 2 };
+/* E8M0_B32: one power-of-two scale shared by 32 consecutive elements (the 1x32 blocks with an E8M0 scale that Sec. 2.1's
+ * footnote attributes to MXFP4), stored as that FP32 power of two for both 16-element halves. */
+enum { ORC_SCALE_FP32 = 0, ORC_SCALE_POW2 = 1, ORC_SCALE_E4M3_TENSOR = 2, ORC_SCALE_E8M0_B32 = 3 };
 enum { ORC_AXIS_ROW = 0, ORC_AXIS_COL = 1 };
 
 /* ---------------------------------------------------------------- codebooks (Sec. 2.1, Sec. 3.1) */
@@ -265,13 +270,14 @@ static float effective_scale(int scale_fmt, float stored_f32, uint8_t stored_byt
 /* One 16-element block.  x: the block's values (BF16 widened to FP32).  Outputs: 16 nibbles, the stored scale
  * (FP32 and, for the E4M3 mode, the byte), and optionally the normalised values y. */
 static void quantize_block(const float x[16], const orc_params *p, uint64_t block_index, uint32_t variant,
-                           uint8_t nib[16], float *scale_f32, uint8_t *scale_byte, float *y_out) {
+                           uint8_t nib[16], float *scale_f32, uint8_t *scale_byte, float *y_out, float amax_shared) {
     float v[16];
     memcpy(v, x, sizeof(v));
     if (p->rht_block == 16) orc_rht16_f32(v, p->sign_mask);
 
     float amax = 0.0f;
     for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+    if (amax_shared >= 0.0f) amax = amax_shared;      /* the scale block is wider than this block: its amax is given */
 
     const float g = (float)orc_gmax(p->grid);
     float s = 0.0f, inv = 0.0f;
@@ -281,7 +287,7 @@ static void quantize_block(const float x[16], const orc_params *p, uint64_t bloc
         if (p->scale_fmt == ORC_SCALE_FP32) {
             s = amax / g;
             inv = g / amax;
-        } else if (p->scale_fmt == ORC_SCALE_POW2) {
+        } else if (p->scale_fmt == ORC_SCALE_POW2 || p->scale_fmt == ORC_SCALE_E8M0_B32) {
             float z = amax / g;
             int e;
             float m = frexpf(z, &e); /* z = m * 2^e, m in [0.5, 1) */
@@ -334,11 +340,12 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int 
                  uint8_t *codes, void *scales, float *y_out) {
     if (!x || !codes || !scales) return -1;
     if (rht_block != 0 && rht_block != 16 && rht_block != 32 && rht_block != 64 && rht_block != 128) return -1;
-    if (grid < 0 || grid > 4 || rounding < 0 || rounding > 1 || scale_fmt < 0 || scale_fmt > 2) return -1;
+    if (grid < 0 || grid > 4 || rounding < 0 || rounding > 1 || scale_fmt < 0 || scale_fmt > 3) return -1;
     int64_t R = (axis == ORC_AXIS_ROW) ? rows : cols; /* output rows   */
     int64_t K = (axis == ORC_AXIS_ROW) ? cols : rows; /* reduction dim */
     if (K % 16 != 0 || R <= 0 || K <= 0) return -1;
     if (rht_block > 16 && K % rht_block != 0) return -1;
+    if (scale_fmt == ORC_SCALE_E8M0_B32 && K % 32 != 0) return -1;
 
     /* RHT blocks wider than the quant block: the whole rht_block-wide chunk is rotated first, then its 16-element
      * blocks are quantized without further rotation. */
@@ -370,11 +377,36 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int 
                 uint32_t u = (uint32_t)h << 16;
                 memcpy(&xb[i], &u, 4);
             }
+            /* 1x32 scale blocks: amax over this 16-element block and its neighbour (kb ^ 1), both after rotation */
+            float amax_shared = -1.0f;
+            if (scale_fmt == ORC_SCALE_E8M0_B32) {
+                float nb[16];
+                int64_t kn = kb ^ 1;
+                for (int i = 0; i < 16; ++i) {
+                    int64_t k = kn * 16 + i;
+                    if (wide) {
+                        nb[i] = chunk[k % rht_block];       /* the neighbour lies in the same rotated chunk */
+                        continue;
+                    }
+                    uint16_t h = (axis == ORC_AXIS_ROW) ? x[o * ld + k] : x[k * ld + o];
+                    uint32_t u = (uint32_t)h << 16;
+                    memcpy(&nb[i], &u, 4);
+                }
+                float own[16];
+                memcpy(own, xb, sizeof(own));
+                if (p.rht_block == 16) {
+                    orc_rht16_f32(nb, p.sign_mask);
+                    orc_rht16_f32(own, p.sign_mask);
+                }
+                amax_shared = 0.0f;
+                for (int i = 0; i < 16; ++i) amax_shared = fmaxf(amax_shared, fmaxf(fabsf(nb[i]), fabsf(own[i])));
+            }
             uint8_t nib[16];
             float sf;
             uint8_t sbyte;
             uint64_t b = (uint64_t)(o * nkb + kb);
-            quantize_block(xb, &p, b, (uint32_t)axis, nib, &sf, &sbyte, y_out ? y_out + (o * K + kb * 16) : NULL);
+            quantize_block(xb, &p, b, (uint32_t)axis, nib, &sf, &sbyte, y_out ? y_out + (o * K + kb * 16) : NULL,
+                           amax_shared);
             for (int j = 0; j < 8; ++j) codes[o * (K / 2) + kb * 8 + j] = (uint8_t)(nib[2 * j] | (nib[2 * j + 1] << 4));
             if (scale_fmt == ORC_SCALE_E4M3_TENSOR) ((uint8_t *)scales)[o * nkb + kb] = sbyte;
             else ((float *)scales)[o * nkb + kb] = sf;

@@ -11,7 +11,7 @@ import pytest
 import torch
 
 import oracle
-from oracle import (AXIS_COL, AXIS_ROW, GRID_E1M2, GRID_E2M1, GRID_E2M1_MAX2, GRID_E2M1_MAX4, GRID_INT4, ROUND_RTNE, ROUND_SR, SCALE_E4M3_TENSOR,
+from oracle import (SCALE_E8M0_B32, AXIS_COL, AXIS_ROW, GRID_E1M2, GRID_E2M1, GRID_E2M1_MAX2, GRID_E2M1_MAX4, GRID_INT4, ROUND_RTNE, ROUND_SR, SCALE_E4M3_TENSOR,
                     SCALE_FP32, SCALE_POW2)
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -529,6 +529,44 @@ def test_pow2_scale_is_the_next_power_of_two_and_is_idempotent():
     again = oracle.quantize(bf16_bits(deq), AXIS_ROW, 0, GRID_INT4, scale_fmt=SCALE_POW2)
     assert np.array_equal(bf16_vals(bf16_bits(deq)), deq)
     assert np.array_equal(again.codes, q.codes) and np.array_equal(again.scales, q.scales)
+
+
+def test_1x32_blocks_with_a_power_of_two_scale():
+    """The MXFP4 block layout of Sec. 2.1's footnote (1 x 32 blocks, E8M0 scale) on the uniform grid: the shared scale is
+    the larger of the two halves' power-of-two scales (rounding up to a power of two is monotone), the half that owns it
+    keeps its POW2 codes, and every code is round-half-even of x / s clipped to the grid (numpy's rint; no RHT, so x / s is
+    an exact division by a power of two)."""
+    bits = _rand_bits(32, 128, 41, 1.7)
+    bits[3, 32:64] = 0                                          # an all-zero 32-block
+    bits[5, 64:80] = 0                                          # a zero half beside a non-zero half
+    x = bf16_vals(bits)
+    for axis in (AXIS_ROW, AXIS_COL):
+        xs = x if axis == AXIS_ROW else x.T
+        a = oracle.quantize(bits, axis, rht_block=0, scale_fmt=SCALE_POW2)
+        b = oracle.quantize(bits, axis, rht_block=0, scale_fmt=SCALE_E8M0_B32)
+        pair = np.maximum(a.scales[:, 0::2], a.scales[:, 1::2])
+        assert np.array_equal(b.scales[:, 0::2], pair) and np.array_equal(b.scales[:, 1::2], pair)
+        nz = b.scales > 0
+        m, e = np.frexp(b.scales[nz])
+        assert np.all(m == 0.5)                                 # powers of two: representable in E8M0
+        s = np.repeat(b.scales.astype(np.float64), 16, axis=1)
+        q = np.zeros_like(xs)
+        np.divide(xs, s, out=q, where=s > 0)
+        q = np.clip(np.rint(q), -7, 7).astype(np.int64)
+        nib = (q & 0xF).astype(np.uint8)
+        assert np.array_equal(b.codes, nib[:, 0::2] | (nib[:, 1::2] << 4))
+        own = np.repeat(a.scales == b.scales, 8, axis=1)        # per code byte: this half owns the shared scale
+        assert np.array_equal(b.codes[own], a.codes[own])
+        assert np.all(np.abs(oracle.dequantize(b) - xs) <= s / 2 + 1e-300)
+    # with the RHT and SR the block indices and draws stay per 16 elements: only the scale is shared
+    a = oracle.quantize(bits, AXIS_ROW, rht_block=16, scale_fmt=SCALE_E8M0_B32, rounding=ROUND_SR, seed_rht=1, seed_sr=2)
+    assert np.array_equal(a.scales[:, 0::2], a.scales[:, 1::2])
+    w = oracle.quantize(bits, AXIS_ROW, rht_block=64, scale_fmt=SCALE_E8M0_B32, seed_rht=1)
+    p = oracle.quantize(bits, AXIS_ROW, rht_block=64, scale_fmt=SCALE_POW2, seed_rht=1)
+    pair = np.maximum(p.scales[:, 0::2], p.scales[:, 1::2])
+    assert np.array_equal(w.scales[:, 0::2], pair) and np.array_equal(w.scales[:, 1::2], pair)
+    with pytest.raises(Exception):
+        oracle.quantize(_rand_bits(16, 48, 1), AXIS_ROW, scale_fmt=SCALE_E8M0_B32)      # 48 is not a multiple of 32
 
 
 def test_e4m3_helpers_round_trip():
