@@ -70,7 +70,15 @@ typedef enum { UFP4_AXIS_ROW = 0, UFP4_AXIS_COL = 1, UFP4_AXIS_BOTH = 2 } ufp4_a
  * power of two, still stored as FP32 (Sec. 4 leaves the scale hierarchy open "depending on hardware efficiency"); it
  * is the format the tensor-core GEMM path folds into its 8-bit operands exactly.  E4M3_TENSOR: an E4M3 byte per
  * block times one FP32 per tensor (the two-level layout Sec. 2.1's footnote attributes to NVFP4). */
-typedef enum { UFP4_SCALE_FP32 = 0, UFP4_SCALE_POW2 = 1, UFP4_SCALE_E4M3_TENSOR = 2 } ufp4_scale_fmt;
+typedef enum {
+    UFP4_SCALE_FP32 = 0, UFP4_SCALE_POW2 = 1, UFP4_SCALE_E4M3_TENSOR = 2,
+    /* One power-of-two scale per 32 consecutive elements: the 1x32 blocks with an E8M0 scale that Sec. 2.1's footnote
+     * attributes to MXFP4, here on any grid.  amax is taken over the 32 (rotated) elements, the scale is the next
+     * power of two >= amax / g_max and is stored, as FP32, for both 16-element halves, so that the GEMM and
+     * diagnostics calls read such a tensor exactly like a POW2 one.  The reduction dimension must be a multiple of 32.
+     * The quantizer serves this format with its plain kernel (see rht_block). */
+    UFP4_SCALE_E8M0_B32 = 3
+} ufp4_scale_fmt;
 
 /* Which training product a GEMM call computes.  All are C = A B^T on k-contiguous operands; the value matters only to
  * the grouped call, where fwd_y / bwd_dx split the rows of A (and C) by group and bwd_dw splits the reduction. */

@@ -16,6 +16,7 @@ GRID_E2M1_MAX4, GRID_E2M1_MAX2 = 3, 4      # range-restricted E2M1 (Sec. 5.4, ma
 ROUND_RTNE, ROUND_SR = 0, 1
 AXIS_ROW, AXIS_COL, AXIS_BOTH = 0, 1, 2
 SCALE_FP32, SCALE_POW2, SCALE_E4M3_TENSOR = 0, 1, 2
+SCALE_E8M0_B32 = 3      # one power-of-two scale per 32 elements (MXFP4's block layout), read by the GEMMs like POW2
 FWD_Y, BWD_DX, BWD_DW = 0, 1, 2
 PATH_AUTO, PATH_EXACT, PATH_TENSOR, PATH_PROMOTE, PATH_SPLIT = 0, 1, 2, 3, 4
 DEV_NONFINITE, DEV_EXP_WINDOW, DEV_WAIT_TIMEOUT = 1, 2, 4

@@ -33,7 +33,7 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
 
 static int check_operand(const ufp4_qtensor *q) {
     if (!q || !q->codes || !q->scales) return UFP4_ERR_NULL;
-    if (q->grid < 0 || q->grid > 4 || q->scale_fmt < 0 || q->scale_fmt > 2) return UFP4_ERR_ENUM;
+    if (q->grid < 0 || q->grid > 4 || q->scale_fmt < 0 || q->scale_fmt > 3) return UFP4_ERR_ENUM;
     if (q->rows < 1 || q->k < 16 || q->k % 16 != 0) return UFP4_ERR_SHAPE;
     if (q->ld_codes_bytes < q->k / 2 || q->ld_codes_bytes % 16 != 0 || q->ld_scales < q->k / 16) return UFP4_ERR_ALIGN;
     if (!aligned_to(q->codes, 16)) return UFP4_ERR_ALIGN;
@@ -105,7 +105,7 @@ extern "C" const char *ufp4_status_string(int status) {
 extern "C" int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t *codes_bytes, size_t *scales_bytes) {
     if (!codes_bytes || !scales_bytes) return UFP4_ERR_NULL;
     if (rows < 1 || k < 16 || k % 16 != 0) return UFP4_ERR_SHAPE;
-    if (scale_fmt < 0 || scale_fmt > 2) return UFP4_ERR_ENUM;
+    if (scale_fmt < 0 || scale_fmt > 3) return UFP4_ERR_ENUM;
     int64_t ld = (k / 2 + 15) / 16 * 16;
     *codes_bytes = (size_t)(rows * ld);
     *scales_bytes = (size_t)(rows * (k / 16) * (scale_fmt == UFP4_SCALE_E4M3_TENSOR ? 1 : 4));
@@ -114,7 +114,7 @@ extern "C" int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t
 
 extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path) {
     if (!A || !B || path == UFP4_PATH_EXACT) return 0;
-    const bool pow2 = A->scale_fmt == UFP4_SCALE_POW2 && B->scale_fmt == UFP4_SCALE_POW2;
+    const bool pow2 = ufp4::is_pow2_fmt(A->scale_fmt) && ufp4::is_pow2_fmt(B->scale_fmt);
     if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
         return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
     // AUTO takes SPLIT, and PROMOTE only where SPLIT does not apply: enough for either

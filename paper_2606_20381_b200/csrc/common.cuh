@@ -39,6 +39,9 @@ constexpr uint32_t kSrCounterTag = 0x53520000u;   // counter word 3 of the SR dr
 // The codebook behind a tensor's nibbles: the range-restricted E2M1 grids store plain E2M1 codes.
 inline int codebook_of(int grid) { return grid > UFP4_GRID_E2M1 ? (int)UFP4_GRID_E2M1 : grid; }
 
+// Scale formats whose stored scales are FP32 powers of two.
+inline bool is_pow2_fmt(int scale_fmt) { return scale_fmt == UFP4_SCALE_POW2 || scale_fmt == UFP4_SCALE_E8M0_B32; }
+
 inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 #define UFP4_CUDA_OK(expr)                                \

@@ -459,7 +459,7 @@ int gemm_tensor_kernel_launches() { return 2; }
 
 bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode) {
     (void)mode;
-    if (A->scale_fmt != UFP4_SCALE_POW2 || B->scale_fmt != UFP4_SCALE_POW2) return false;
+    if (!is_pow2_fmt(A->scale_fmt) || !is_pow2_fmt(B->scale_fmt)) return false;
     if (K % 16 != 0 || M < 1 || N < 1) return false;
     if (A->rows > 0x7FFFFFFF || B->rows > 0x7FFFFFFF || K > 0x7FFFFFFF) return false;
     return true;

@@ -68,6 +68,37 @@ def test_wide_rht_blocks(rht_block, shape, grid, rounding, scale_fmt):
     run_both(x, ufp4.AXIS_BOTH, **kw)
 
 
+@pytest.mark.parametrize("rht_block", [0, 16, 64])
+@pytest.mark.parametrize("grid", [ufp4.GRID_INT4, ufp4.GRID_E1M2, ufp4.GRID_E2M1, ufp4.GRID_E2M1_MAX4])
+@pytest.mark.parametrize("rounding", [ufp4.ROUND_RTNE, ufp4.ROUND_SR])
+def test_1x32_blocks_with_a_power_of_two_scale(rht_block, grid, rounding):
+    """The MXFP4 block layout (1 x 32 blocks, E8M0 scale; Sec. 2.1's footnote): both layouts bit-equal to the oracle on a
+    ragged multi-tile matrix, and the two halves of every 32-block share their scale."""
+    x = inputs.spiky_normal(320, 192, seed=17)
+    row, col = run_both(x, ufp4.AXIS_BOTH, rht_block=rht_block, grid=grid, rounding=rounding,
+                        scale_fmt=ufp4.SCALE_E8M0_B32, seed_rht=5, seed_sr=9)
+    for q in (row, col):
+        assert torch.equal(q.scales[:, 0::2], q.scales[:, 1::2])
+
+
+def test_1x32_blocks_feed_every_gemm_path_as_power_of_two_scales():
+    from helpers import assert_gemm_close
+    X = inputs.heavy_tailed_activations(200, 256, seed=81)
+    W = inputs.normal_bf16(136, 256, 0.02, seed=82)
+    kw = dict(rht_block=16, scale_fmt=ufp4.SCALE_E8M0_B32, seed_rht=3)
+    A, _ = ufp4.quantize(X.cuda(), axis=ufp4.AXIS_ROW, **kw)
+    B, _ = ufp4.quantize(W.cuda(), axis=ufp4.AXIS_ROW, **kw)
+    ref, S = oracle.gemm(oracle_quantize(X, oracle.AXIS_ROW, **kw), oracle_quantize(W, oracle.AXIS_ROW, **kw))
+    assert ufp4.gemm_path_name(A, B) == "tensor"
+    for path in (ufp4.PATH_AUTO, ufp4.PATH_TENSOR, ufp4.PATH_SPLIT, ufp4.PATH_PROMOTE, ufp4.PATH_EXACT):
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        out = ufp4.gemm(A, B, path=path, dev_status=status)
+        assert int(status.item()) == 0
+        assert_gemm_close(out.cpu().numpy(), ref, S, f"path {path}")
+    with pytest.raises(ufp4.Ufp4Error):                     # 48 columns: not a multiple of 32
+        ufp4.quantize(inputs.normal_bf16(32, 48, 1.0, seed=1).cuda(), axis=ufp4.AXIS_ROW, scale_fmt=ufp4.SCALE_E8M0_B32)
+
+
 def test_wide_rht_single_axis_and_shape_rules():
     x = inputs.normal_bf16(48, 256, 1.0, seed=3)            # 48 rows: the row variant alone takes any row count
     run_both(x, ufp4.AXIS_ROW, rht_block=128, seed_rht=2)
