@@ -77,7 +77,7 @@ constexpr int kDecodeThreads = 256;
 
 // A CTA decodes 256 / TPR rows with TPR threads (32..256) on each: short rows keep a warp per row, long rows are
 // spread over more threads so that the grid has many more warps than the GPU has slots (no idle tail).
-template <int TPR>
+template <int TPR, bool OWN>
 __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const DecodeParams P) {
     constexpr int kRowsPerCta = kDecodeThreads / TPR;
     if ((int64_t)blockIdx.x == P.tbl_cta) {
@@ -110,28 +110,54 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
         pf[u] = in ? (int)(__float_as_uint(__ldg(sptr + u * TPR)) >> 23) : 0;   // scales are non-negative: no sign bit
     }
 
-    // largest block exponent field of the row (power-of-two scales: the exponent field is the scale; 0 = zero block).
-    // Every warp of a row scans the whole row's scales (a 32nd of the traffic; the repeats hit in cache): no shared
-    // memory and no CTA barrier, so that this kernel's CTAs fit beside a resident product-kernel CTA on the same SM.
-    uint32_t fmax = 0u;
-    if (active) {
-        // eight loads in flight per thread: the row's scales are the first touch of DRAM, and a warp issues in order
-        const float *srow0 = sptr - t;
-        int kb = lane;
-        for (; kb + 7 * 32 < nkb; kb += 8 * 32) {
-            uint32_t b[8];
+    // largest block exponent field of the row (power-of-two scales: the exponent field is the scale; 0 = zero block),
+    // eight loads in flight per thread.  OWN (rows spread over four or eight warps): a thread scans the scales of its own
+    // blocks only, the lanes of a warp combine by shuffles and the warps of a row through shared memory.  Otherwise
+    // (one or two warps per row) every warp scans the whole row (the repeats hit in cache) and no barrier is needed.
+    int fmax = 0;
+    if (OWN) {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) b[u] = __float_as_uint(__ldg(srow0 + kb + u * 32));
+        for (int u = 0; u < kPre; ++u) fmax = max(fmax, pf[u]);
+        if (active) {
+            int kb = t + kPre * TPR;
+            for (; kb + 7 * TPR < nkb; kb += 8 * TPR) {
+                uint32_t b[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) fmax = max(fmax, b[u]);
+                for (int u = 0; u < 8; ++u) b[u] = __float_as_uint(__ldg(sptr + (kb - t) + u * TPR));
+#pragma unroll
+                for (int u = 0; u < 8; ++u) fmax = max(fmax, (int)(b[u] >> 23));
+            }
+            for (; kb < nkb; kb += TPR) fmax = max(fmax, (int)(__float_as_uint(__ldg(sptr + (kb - t))) >> 23));
         }
-        for (; kb < nkb; kb += 32) fmax = max(fmax, __float_as_uint(__ldg(srow0 + kb)));
-    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) fmax = max(fmax, __shfl_xor_sync(0xFFFFFFFFu, fmax, o));
+        for (int o = 16; o > 0; o >>= 1) fmax = max(fmax, __shfl_xor_sync(0xFFFFFFFFu, fmax, o));
+        __shared__ int wmax[kDecodeThreads / 32];
+        if (lane == 0) wmax[threadIdx.x >> 5] = fmax;
+        __syncthreads();
+        const int w0 = (threadIdx.x / TPR) * (TPR / 32);
+#pragma unroll
+        for (int i = 0; i < TPR / 32; ++i) fmax = max(fmax, wmax[w0 + i]);
+    } else {
+        uint32_t fm = 0u;
+        if (active) {
+            const float *srow0 = sptr - t;
+            int kb = lane;
+            for (; kb + 7 * 32 < nkb; kb += 8 * 32) {
+                uint32_t b[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) b[u] = __float_as_uint(__ldg(srow0 + kb + u * 32));
+#pragma unroll
+                for (int u = 0; u < 8; ++u) fm = max(fm, b[u]);
+            }
+            for (; kb < nkb; kb += 32) fm = max(fm, __float_as_uint(__ldg(srow0 + kb)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) fm = max(fm, __shfl_xor_sync(0xFFFFFFFFu, fm, o));
+        fmax = (int)(fm >> 23);
+    }
     if (!active) return;
     // biased exponent field of the row's reference 2^eref, eref = emax - kDMax (an all-zero row takes eref = 0)
-    const int fref = fmax == 0u ? 127 : (int)(fmax >> 23) - kDMax;
+    const int fref = fmax == 0 ? 127 : fmax - kDMax;
     if (t == 0) {
         // unit * 2^eref as two exact factors (fref may be below the smallest normal exponent field)
         const float unit = O.grid == UFP4_GRID_INT4 ? 1.0f : (O.grid == UFP4_GRID_E1M2 ? 0.25f : 0.5f);
@@ -504,10 +530,12 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     const int64_t decode_ctas = D.tbl_cta + (mode == 1 && cg == 2 ? 1 : 0);
     if (decode_ctas > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     const unsigned dg = (unsigned)decode_ctas;
-    if (tpr == 32) decode_rows_kernel<32><<<dg, kDecodeThreads, 0, st>>>(D);
-    else if (tpr == 64) decode_rows_kernel<64><<<dg, kDecodeThreads, 0, st>>>(D);
-    else if (tpr == 128) decode_rows_kernel<128><<<dg, kDecodeThreads, 0, st>>>(D);
-    else decode_rows_kernel<256><<<dg, kDecodeThreads, 0, st>>>(D);
+    // rows spread over four or eight warps: each thread scans only its own blocks' scales and the warps combine
+    // through shared memory; with one or two warps per row every warp scans the whole row (no barrier; measured faster)
+    if (tpr == 32) decode_rows_kernel<32, false><<<dg, kDecodeThreads, 0, st>>>(D);
+    else if (tpr == 64) decode_rows_kernel<64, false><<<dg, kDecodeThreads, 0, st>>>(D);
+    else if (tpr == 128) decode_rows_kernel<128, true><<<dg, kDecodeThreads, 0, st>>>(D);
+    else decode_rows_kernel<256, true><<<dg, kDecodeThreads, 0, st>>>(D);
     if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
 
     CUtensorMap tmA, tmB;
