@@ -110,23 +110,46 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
                            ? static_cast<const void *>(static_cast<const uint8_t *>(O.scales) + r_safe * O.lds)
                            : static_cast<const void *>(static_cast<const float *>(O.scales) + r_safe * O.lds);
 
-    // largest block scale of the row (scales are non-negative: their bit patterns order like their values).  Every warp
-    // of a row scans the whole row's scales (the repeats hit in cache): no shared memory and no CTA barrier, so that
-    // this kernel's CTAs fit beside a resident product-kernel CTA on the same SM.
+    // largest block scale of the row (scales are non-negative: their bit patterns order like their values), eight loads
+    // in flight per thread.  One or two warps per row: every warp scans the whole row (the repeats hit in cache) and no
+    // barrier is needed.  Four or eight warps per row: a thread scans the scales of its own blocks only and the warps
+    // combine through shared memory.
     uint32_t smax = 0u;
-    if (active) {
-        int kb = lane;
-        for (; kb + 7 * 32 < nkb; kb += 8 * 32) {
-            float s[8];
+    if (TPR >= 128) {
+        if (active) {
+            int kb = t;
+            for (; kb + 7 * TPR < nkb; kb += 8 * TPR) {
+                float s[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) s[u] = split_scale_of(O, srow, kb + u * 32, ts);
+                for (int u = 0; u < 8; ++u) s[u] = split_scale_of(O, srow, kb + u * TPR, ts);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) smax = max(smax, __float_as_uint(s[u]));
+                for (int u = 0; u < 8; ++u) smax = max(smax, __float_as_uint(s[u]));
+            }
+            for (; kb < nkb; kb += TPR) smax = max(smax, __float_as_uint(split_scale_of(O, srow, kb, ts)));
         }
-        for (; kb < nkb; kb += 32) smax = max(smax, __float_as_uint(split_scale_of(O, srow, kb, ts)));
-    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) smax = max(smax, __shfl_xor_sync(0xFFFFFFFFu, smax, o));
+        for (int o = 16; o > 0; o >>= 1) smax = max(smax, __shfl_xor_sync(0xFFFFFFFFu, smax, o));
+        __shared__ uint32_t wmax[kSDecodeThreads / 32];
+        if (lane == 0) wmax[threadIdx.x >> 5] = smax;
+        __syncthreads();
+        const int w0 = (threadIdx.x / TPR) * (TPR / 32);
+#pragma unroll
+        for (int i = 0; i < TPR / 32; ++i) smax = max(smax, wmax[w0 + i]);
+    } else {
+        if (active) {
+            int kb = lane;
+            for (; kb + 7 * 32 < nkb; kb += 8 * 32) {
+                float s[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) s[u] = split_scale_of(O, srow, kb + u * 32, ts);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) smax = max(smax, __float_as_uint(s[u]));
+            }
+            for (; kb < nkb; kb += 32) smax = max(smax, __float_as_uint(split_scale_of(O, srow, kb, ts)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) smax = max(smax, __shfl_xor_sync(0xFFFFFFFFu, smax, o));
+    }
     if (!active) return;
 
     // Reference 2^(e - 11), e the exponent of the largest scale: the largest normalised scale lies in [2^11, 2^12) and
