@@ -21,11 +21,11 @@ def _bf16(a):
 def test_quantizer_random_cases(seed):
     """Ten cases per seed: R, C up to 640, RHT blocks of 0 / 16 / 32 / 64 / 128; plain normal, per-row scaling over 2^+-110 (subnormal and near-overflow
     blocks), per-element scaling over 2^+-30, 70 % zeros, quarter-integer values (exact rounding ties); all five grids
-    (the range-restricted E2M1 variants included)."""
+    (the range-restricted E2M1 variants included); FP32, power-of-two and 1 x 32 power-of-two scales."""
     rng = np.random.default_rng(1000 + seed)
     for _ in range(10):
         rht = int(rng.choice([0, 16, 16, 32, 64, 128]))
-        unit = max(16, rht)                                         # both reduction dimensions hold whole RHT blocks
+        unit = max(32, rht)                                         # whole RHT blocks and whole 1 x 32 scale blocks
         R, C = unit * int(rng.integers(1, 640 // unit + 1)), unit * int(rng.integers(1, 640 // unit + 1))
         x = rng.standard_normal((R, C)).astype(np.float32)
         mode = int(rng.integers(0, 5))
@@ -39,7 +39,7 @@ def test_quantizer_random_cases(seed):
             x = np.round(x * 4) / 4 * np.exp2(rng.integers(-5, 5))
         xt = _bf16(x)
         kw = dict(rht_block=rht, grid=int(rng.integers(0, 5)), rounding=int(rng.integers(0, 2)),
-                  scale_fmt=int(rng.integers(0, 2)), seed_rht=int(rng.integers(0, 1 << 40)), seed_sr=int(rng.integers(0, 1 << 40)))
+                  scale_fmt=int(rng.choice([0, 1, 3])), seed_rht=int(rng.integers(0, 1 << 40)), seed_sr=int(rng.integers(0, 1 << 40)))
         status = torch.zeros(1, dtype=torch.int32, device="cuda")
         row, col = ufp4.quantize(xt.cuda(), axis=ufp4.AXIS_BOTH, dev_status=status, **kw)
         what = f"R {R} C {C} mode {mode} {kw}"
