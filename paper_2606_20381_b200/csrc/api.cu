@@ -86,7 +86,7 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
 
 }  // namespace ufp4
 
-extern "C" int ufp4_version(void) { return 100; }
+extern "C" int ufp4_version(void) { return 200; }
 
 extern "C" const char *ufp4_status_string(int status) {
     switch (status) {
