@@ -193,6 +193,18 @@ def test_nonfinite_input_sets_the_status_bit():
     status.zero_()
     ufp4.quantize(x.cuda(), axis=ufp4.AXIS_BOTH, rht_block=0, dev_status=status)
     assert int(status.item()) & ufp4.DEV_NONFINITE
+    # the plain kernel (wider RHT blocks, 1 x 32 scale blocks) reports it too; finite inputs leave the word clear
+    x = inputs.normal_bf16(128, 128, 1.0, seed=13)
+    for kw in (dict(rht_block=64), dict(rht_block=16, scale_fmt=ufp4.SCALE_E8M0_B32), dict(rht_block=0, scale_fmt=ufp4.SCALE_E8M0_B32)):
+        status.zero_()
+        ufp4.quantize(x.cuda(), axis=ufp4.AXIS_BOTH, dev_status=status, **kw)
+        assert int(status.item()) == 0
+        for bad in (float("inf"), float("nan")):
+            y = x.clone()
+            y[100, 37] = bad
+            status.zero_()
+            ufp4.quantize(y.cuda(), axis=ufp4.AXIS_BOTH, dev_status=status, **kw)
+            assert int(status.item()) & ufp4.DEV_NONFINITE, (kw, bad)
 
 
 def test_batched_weights_stack_along_rows():
