@@ -72,7 +72,7 @@ def lib():
         L.orc_bin_bias.restype = None
         L.orc_bin_bias.argtypes = [p, p, i64, i32, p, p]
         L.orc_diagnose.restype = None
-        L.orc_diagnose.argtypes = [p, i64, i64, i64, p, i64, p, i64, i32, i32, C.c_uint32, p]
+        L.orc_diagnose.argtypes = [p, i64, i64, i64, p, i64, p, i64, i32, i32, u64, p]
         L.orc_b_eff.restype = f64
         L.orc_b_eff.argtypes = [p]
         _lib = L
@@ -253,7 +253,7 @@ def diagnose(x_u16: np.ndarray, q: QTensor, rht_block: int, seed_rht: int) -> di
     scales = np.ascontiguousarray(q.scales, dtype=np.float32)
     out = np.zeros(19, dtype=np.float64)
     lib().orc_diagnose(_ptr(x), rows, cols, cols, _ptr(codes), cols // 2, _ptr(scales), cols // 16, q.grid, rht_block,
-                       int(rht_sign_mask(seed_rht)), _ptr(out))
+                       seed_rht, _ptr(out))
     return diagnostics_from_sums(out)
 
 

@@ -494,8 +494,9 @@ void orc_bin_bias(const float *y, const uint8_t *codes, int64_t n, int grid, int
 
 /* ---------------------------------------------------------------- tensor diagnostics (Sec. 3.2 Eq. 3, Sec. 3.3 Eq. 6-7) */
 
-/* For the row variant (codes, FP32 scales) of the BF16 matrix x [rows][cols], with x' = x H'_16 per 16-block
- * (rht_block == 16; FP32 butterflies as in the quantizer) or x' = x (rht_block == 0) and xq = level * scale:
+/* For the row variant (codes, FP32 scales) of the BF16 matrix x [rows][cols], with x' = x H'_n per n-element chunk
+ * (rht_block n = 16, 32, 64 or 128; FP32 butterflies as in the quantizer) or x' = x (rht_block == 0) and
+ * xq = level * scale:
  *   out[0] = sum x'^2, out[1] = sum (xq - x')^2, out[2] = sum xq x'            (Eq. 3: alpha = out[2] / out[0];
  *                                                                               Sec. 3.3: NMSE = out[1] / out[0])
  *   out[3 + i]  = number of elements whose code has magnitude level i           (Eq. 6: p_i = out[3 + i] / n)
@@ -503,17 +504,32 @@ void orc_bin_bias(const float *y, const uint8_t *codes, int64_t n, int grid, int
  *                                                                               block contributes 0 to it)
  * All sums in FP64, elements in storage order. */
 void orc_diagnose(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, const uint8_t *codes, int64_t ld_codes,
-                  const float *scales, int64_t ld_scales, int grid, int rht_block, uint32_t sign_mask, double out[19]) {
+                  const float *scales, int64_t ld_scales, int grid, int rht_block, uint64_t seed_rht, double out[19]) {
     const double *L = levels_of(grid);
+    const uint32_t sign_mask = orc_rht_sign_mask(seed_rht);
+    uint32_t signs[4];
+    orc_rht_signs(seed_rht, signs);
+    float chunk[128];
     for (int i = 0; i < 19; ++i) out[i] = 0.0;
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t b = 0; b < cols / 16; ++b) {
             float v[16];
-            for (int i = 0; i < 16; ++i) {
-                uint32_t bits = (uint32_t)x[r * ld + 16 * b + i] << 16;
-                memcpy(&v[i], &bits, 4);
+            if (rht_block > 16) {
+                if ((16 * b) % rht_block == 0) {        /* a new chunk: rotate all of it */
+                    for (int i = 0; i < rht_block; ++i) {
+                        uint32_t bits = (uint32_t)x[r * ld + 16 * b + i] << 16;
+                        memcpy(&chunk[i], &bits, 4);
+                    }
+                    orc_rht_f32(chunk, rht_block, signs);
+                }
+                memcpy(v, chunk + (16 * b) % rht_block, sizeof(v));
+            } else {
+                for (int i = 0; i < 16; ++i) {
+                    uint32_t bits = (uint32_t)x[r * ld + 16 * b + i] << 16;
+                    memcpy(&v[i], &bits, 4);
+                }
+                if (rht_block == 16) orc_rht16_f32(v, sign_mask);
             }
-            if (rht_block == 16) orc_rht16_f32(v, sign_mask);
             const double s = (double)scales[r * ld_scales + b];
             for (int i = 0; i < 16; ++i) {
                 const int64_t e = 16 * b + i;

@@ -730,3 +730,19 @@ def test_diagnostics_against_a_matrix_formulation():
     n_free = 256 * 256 * 15 / 16
     assert abs(d["sums"][1] / n_free - 1 / 12) < 0.003      # BF16 inputs are themselves on a fine grid: still 1/12
     assert np.nanmax(np.abs(d["bias"][1:7])) < 0.01         # symmetric bins: no bias (Sec. 3.1)
+
+
+def test_diagnostics_with_a_wide_rht_block_equal_those_of_the_pre_rotated_tensor():
+    """RHT block 64 on entries in {-1, 0, 1} (the rotated tensor is BF16-exact, 1/8 being a power of two): the sums of
+    orc_diagnose must be those of the pre-rotated tensor quantized without rotation; the rotation preserves the energy."""
+    rng = np.random.default_rng(64)
+    x = rng.integers(-1, 2, size=(48, 256)).astype(np.float32)
+    bits = bf16_bits(x)
+    signs = oracle.rht_signs(5)
+    rot = np.stack([np.concatenate([oracle.rht_f32(r[c:c + 64], 64, signs) for c in range(0, r.size, 64)]) for r in x])
+    pre = bf16_bits(rot)
+    for grid in (GRID_INT4, GRID_E2M1):
+        a = oracle.diagnose(bits, oracle.quantize(bits, AXIS_ROW, rht_block=64, grid=grid, seed_rht=5), 64, 5)
+        b = oracle.diagnose(pre, oracle.quantize(pre, AXIS_ROW, rht_block=0, grid=grid), 0, 5)
+        assert np.array_equal(a["sums"], b["sums"]) and np.array_equal(a["count"], b["count"])
+        assert a["sums"][0] == float(np.sum(x.astype(np.float64) ** 2))
