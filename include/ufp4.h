@@ -219,7 +219,8 @@ int ufp4_gemm_grouped(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
 
 /*
  * Tensor diagnostics of Sec. 3 on a BF16 matrix x [rows][cols] and its row variant q_row (FP32 or POW2 scales), with
- * x' = x H'_16 per 16-block for rht_block == 16 (the quantizer's FP32 butterflies) or x' = x for rht_block == 0, and
+ * x' = x H'_n per n-element chunk for rht_block n = 16, 32, 64 or 128 (the quantizer's FP32 butterflies; cols must be a
+ * multiple of n) or x' = x for rht_block == 0, and
  * xq = level * scale.  dev_out (device, 19 doubles) receives
  *   [0] sum x'^2   [1] sum (xq - x')^2   [2] sum xq x'      -> alpha = [2] / [0] (Eq. 3), NMSE = [1] / [0] (Sec. 3.3;
  *                                                              Delta SQNR of Eq. 7 is 10 log10 of the ratio of two NMSEs)

@@ -20,7 +20,9 @@ struct DiagParams {
     int64_t ldc, lds;
     int grid, rht;
     int load256;                   // x and its row pitch are 32-byte aligned: 256-bit loads
-    uint32_t sign_mask;
+    uint32_t signs[4];             // bit i of the 128: eps_i = -1 (the first 16 bits serve the 16-point transform)
+    int xb;                        // log2(rht_block / 16): butterfly stages that pair 16-element blocks
+    float norm;                    // 1/4, or RN(1 / sqrt(rht_block)) for the wider blocks
     double *partials;              // [gridDim.x][kDiagSums]
 };
 
@@ -36,8 +38,6 @@ __device__ __forceinline__ void diag_butterflies(float (&v)[16]) {
             }
         }
     }
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(v[i], 0.25f);
 }
 
 template <int GRID>
@@ -50,7 +50,14 @@ __global__ void __launch_bounds__(kDiagThreads) diagnose_kernel(const DiagParams
 #pragma unroll
     for (int k = 0; k < 8; ++k) { cnt[k] = 0; lvl[k][threadIdx.x] = 0.0f; }
 
-    for (int64_t blk = (int64_t)blockIdx.x * kDiagThreads + threadIdx.x; blk < nblk; blk += (int64_t)gridDim.x * kDiagThreads) {
+    // warp-uniform trip count: with an RHT block wider than 16 the eight (or fewer) neighbouring lanes that hold one
+    // block's 16-element pieces exchange registers, so every lane of a warp runs every iteration (a lane past the end
+    // works on zeros and adds nothing); rows hold whole RHT blocks, so a group of lanes never straddles two rows
+    const int lane0 = threadIdx.x & ~31;
+    for (int64_t base = (int64_t)blockIdx.x * kDiagThreads + lane0; base < nblk; base += (int64_t)gridDim.x * kDiagThreads) {
+        const int64_t blk_raw = base + (threadIdx.x & 31);
+        const bool valid = blk_raw < nblk;
+        const int64_t blk = valid ? blk_raw : 0;
         const int64_t r = blk / bpr, b = blk - r * bpr;
         const uint4 *src = reinterpret_cast<const uint4 *>(P.x + r * P.ld + 16 * b);
         uint4 d0, d1;
@@ -62,7 +69,7 @@ __global__ void __launch_bounds__(kDiagThreads) diagnose_kernel(const DiagParams
             d1 = __ldg(src + 1);
         }
         const uint2 cw = __ldg(reinterpret_cast<const uint2 *>(P.codes + r * P.ldc + 8 * b));
-        const float s = __ldg(P.scales + r * P.lds + b);
+        const float s = valid ? __ldg(P.scales + r * P.lds + b) : 0.0f;
         const uint32_t w[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
         float v[16];
 #pragma unroll
@@ -71,10 +78,24 @@ __global__ void __launch_bounds__(kDiagThreads) diagnose_kernel(const DiagParams
             v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
         }
         if (P.rht) {
+            const int j = (int)b & ((1 << P.xb) - 1);              // this block's place inside its RHT block
+            const uint32_t sb = P.signs[j >> 1] >> (16 * (j & 1));
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(__float_as_uint(v[i]) ^ (((P.sign_mask >> i) & 1u) << 31));
+            for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(__float_as_uint(v[i]) ^ (((sb >> i) & 1u) << 31));
             diag_butterflies(v);
+            for (int st = 0; st < P.xb; ++st) {
+                const int m = 1 << st;
+                const bool upper = (j & m) != 0;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float o = __shfl_xor_sync(0xFFFFFFFFu, v[i], m);
+                    v[i] = upper ? __fsub_rn(o, v[i]) : __fadd_rn(v[i], o);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(v[i], P.norm);
         }
+        if (!valid) continue;                                      // uniform exchanges are done: nothing to add
         const float inv_s = s > 0.0f ? 1.0f / s : 0.0f;          // t only feeds an average: a rounded reciprocal is fine
         uint64_t hist = 0;                                      // one byte per level: this block's counts
         float bxx = 0.0f, bee = 0.0f, bxq = 0.0f;               // the block's three sums in FP32 (16 terms), FP64 across blocks
@@ -154,7 +175,8 @@ extern "C" int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t 
                              uint64_t seed_rht, double *dev_out, void *workspace, size_t workspace_bytes, void *stream) {
     if (!x || !q_row || !q_row->codes || !q_row->scales || !dev_out || !workspace) return UFP4_ERR_NULL;
     if (rows < 1 || cols < 16 || cols % 16 != 0 || ld < cols || q_row->rows != rows || q_row->k != cols) return UFP4_ERR_SHAPE;
-    if (rht_block != 0 && rht_block != 16) return UFP4_ERR_UNSUPPORTED;
+    if (rht_block != 0 && rht_block != 16 && rht_block != 32 && rht_block != 64 && rht_block != 128) return UFP4_ERR_UNSUPPORTED;
+    if (rht_block > 16 && cols % rht_block != 0) return UFP4_ERR_SHAPE;
     if (q_row->grid < 0 || q_row->grid > 4) return UFP4_ERR_ENUM;
     if (q_row->scale_fmt == UFP4_SCALE_E4M3_TENSOR) return UFP4_ERR_UNSUPPORTED;
     if (!ufp4::aligned_to(x, 16) || (ld * 2) % 16 != 0 || !ufp4::aligned_to(q_row->codes, 8) || q_row->ld_codes_bytes % 8 != 0 ||
@@ -167,9 +189,11 @@ extern "C" int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t 
     P.codes = static_cast<const uint8_t *>(q_row->codes);
     P.scales = static_cast<const float *>(q_row->scales);
     P.ldc = q_row->ld_codes_bytes; P.lds = q_row->ld_scales;
-    P.grid = ufp4::codebook_of(q_row->grid); P.rht = rht_block == 16;
+    P.grid = ufp4::codebook_of(q_row->grid); P.rht = rht_block != 0;
+    P.xb = rht_block == 32 ? 1 : (rht_block == 64 ? 2 : (rht_block == 128 ? 3 : 0));
+    P.norm = rht_block <= 16 ? 0.25f : (float)(1.0 / sqrt((double)rht_block));
     P.load256 = ufp4::aligned_to(x, 32) && ld % 16 == 0;
-    P.sign_mask = ufp4_rht_sign_mask(seed_rht);
+    ufp4_rht_signs(seed_rht, P.signs);
     P.partials = static_cast<double *>(workspace);
     const int64_t nblk = rows * (cols / 16);
     int64_t ctas = (nblk + ufp4::kDiagThreads - 1) / ufp4::kDiagThreads;

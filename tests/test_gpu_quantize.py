@@ -272,6 +272,16 @@ def test_tensor_diagnostics_agree_with_the_oracle():
             assert np.allclose(got["bias"].numpy(), rb, atol=2e-5, equal_nan=True)
             again = diagnostics.tensor_diagnostics(x.cuda(), row, rht, 1)
             assert torch.equal(again["sums"], got["sums"])
+    # RHT blocks wider than the quant block (cols = 1040 is no multiple of them: a 1024-column slice)
+    xs = x[:, :1024].contiguous()
+    xsb = inputs.bf16_bits(xs)
+    for rht in (32, 64, 128):
+        row, _ = ufp4.quantize(xs.cuda(), axis=ufp4.AXIS_ROW, rht_block=rht, seed_rht=1)
+        got = diagnostics.tensor_diagnostics(xs.cuda(), row, rht, 1)
+        ref = oracle.diagnose(xsb, oracle_quantize(xs, oracle.AXIS_ROW, rht_block=rht, seed_rht=1), rht, 1)
+        assert np.array_equal(got["count"].numpy(), ref["count"])
+        assert np.allclose(got["sums"].numpy()[:3], ref["sums"][:3], rtol=1e-6)
+        assert np.allclose(got["bias"].numpy(), ref["bias"], atol=2e-5, equal_nan=True)
     # direction of the effect the paper describes: after RHT the E2M1 levels 2 and 4 shrink, the uniform grid does not
     row, _ = ufp4.quantize(x.cuda(), axis=ufp4.AXIS_ROW, rht_block=16, grid=ufp4.GRID_E2M1, seed_rht=1)
     _, b = diagnostics.per_bin_bias(x.cuda(), row, 16, 1)
