@@ -111,9 +111,10 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
     }
 
     // largest block exponent field of the row (power-of-two scales: the exponent field is the scale; 0 = zero block),
-    // eight loads in flight per thread.  OWN (rows spread over four or eight warps): a thread scans the scales of its own
-    // blocks only, the lanes of a warp combine by shuffles and the warps of a row through shared memory.  Otherwise
-    // (one or two warps per row) every warp scans the whole row (the repeats hit in cache) and no barrier is needed.
+    // eight loads in flight per thread.  OWN (a warp per row, or rows spread over four or eight warps): a thread scans
+    // the scales of its own blocks only (the first of them are already in registers), the lanes of a warp combine by
+    // shuffles and the warps of a row through shared memory.  Otherwise (two warps per row) both warps scan the whole
+    // row (the repeats hit in cache) and no barrier is needed.
     int fmax = 0;
     if (OWN) {
 #pragma unroll
@@ -131,12 +132,14 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) fmax = max(fmax, __shfl_xor_sync(0xFFFFFFFFu, fmax, o));
-        __shared__ int wmax[kDecodeThreads / 32];
-        if (lane == 0) wmax[threadIdx.x >> 5] = fmax;
-        __syncthreads();
-        const int w0 = (threadIdx.x / TPR) * (TPR / 32);
+        if (TPR > 32) {
+            __shared__ int wmax[kDecodeThreads / 32];
+            if (lane == 0) wmax[threadIdx.x >> 5] = fmax;
+            __syncthreads();
+            const int w0 = (threadIdx.x / TPR) * (TPR / 32);
 #pragma unroll
-        for (int i = 0; i < TPR / 32; ++i) fmax = max(fmax, wmax[w0 + i]);
+            for (int i = 0; i < TPR / 32; ++i) fmax = max(fmax, wmax[w0 + i]);
+        }
     } else {
         uint32_t fm = 0u;
         if (active) {
@@ -530,9 +533,9 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     const int64_t decode_ctas = D.tbl_cta + (mode == 1 && cg == 2 ? 1 : 0);
     if (decode_ctas > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     const unsigned dg = (unsigned)decode_ctas;
-    // rows spread over four or eight warps: each thread scans only its own blocks' scales and the warps combine
-    // through shared memory; with one or two warps per row every warp scans the whole row (no barrier; measured faster)
-    if (tpr == 32) decode_rows_kernel<32, false><<<dg, kDecodeThreads, 0, st>>>(D);
+    // a warp per row, or rows spread over four or eight warps: each thread scans only its own blocks' scales (the warps of
+    // a row combine through shared memory); with two warps per row both scan the whole row (no barrier; measured faster)
+    if (tpr == 32) decode_rows_kernel<32, true><<<dg, kDecodeThreads, 0, st>>>(D);
     else if (tpr == 64) decode_rows_kernel<64, false><<<dg, kDecodeThreads, 0, st>>>(D);
     else if (tpr == 128) decode_rows_kernel<128, true><<<dg, kDecodeThreads, 0, st>>>(D);
     else decode_rows_kernel<256, true><<<dg, kDecodeThreads, 0, st>>>(D);
