@@ -351,6 +351,45 @@ def test_sr_expectation_through_the_quantizer():
         assert not np.array_equal(q.codes, q2.codes) and np.array_equal(q.codes, q3.codes)
 
 
+def test_sr_draws_are_keyed_by_block_index_and_variant():
+    """Which random bytes a block sees: block b = o * (K/16) + kb of the variant's own scales array (o = output row,
+    kb = block along the reduction axis), variant word 0 for the row layout and 1 for the col layout, element j of the
+    block taking byte j.  The codes of a small tensor are rebuilt here from sr_bytes() and round_sr() alone, with the
+    scale arithmetic written out in numpy; a transposed, shifted or swapped index in the quantizer would change them."""
+    rows, cols = 32, 48
+    rng = np.random.default_rng(77)
+    bits = bf16_bits(rng.standard_normal((rows, cols)) * np.exp(rng.standard_normal((rows, 1))))
+    x = bf16_vals(bits).astype(np.float32)
+    seed_sr = 0x1234567_89ABCDEF
+    for axis, variant in ((AXIS_ROW, 0), (AXIS_COL, 1)):
+        v = x if axis == AXIS_ROW else np.ascontiguousarray(x.T)      # [output row o][reduction index]
+        R, K = v.shape
+        nkb = K // 16
+        for grid, gmax in ((GRID_INT4, 7.0), (GRID_E2M1, 6.0)):
+            q = oracle.quantize(bits, axis, rht_block=0, grid=grid, rounding=ROUND_SR, seed_sr=seed_sr)
+            L = oracle.levels(grid)
+            expect = np.zeros((R, K), dtype=np.int64)
+            for o in range(R):
+                for kb in range(nkb):
+                    blk = v[o, 16 * kb:16 * kb + 16]
+                    amax = np.float32(np.max(np.abs(blk)))
+                    inv = np.float32(gmax) / amax
+                    y = (blk * inv).astype(np.float32)
+                    r = oracle.sr_bytes(seed_sr, o * nkb + kb, variant)
+                    for j in range(16):
+                        idx = oracle.round_sr(abs(float(y[j])), grid, int(r[j]))
+                        if grid == GRID_INT4:
+                            expect[o, 16 * kb + j] = (-idx if y[j] < 0 else idx) & 0xF
+                        else:
+                            expect[o, 16 * kb + j] = 0 if idx == 0 else ((8 if y[j] < 0 else 0) | idx)
+            got = np.stack([q.codes & 0xF, q.codes >> 4], axis=-1).reshape(R, K)
+            assert np.array_equal(got, expect)
+            # the mapping matters on this input: the neighbouring block's bytes or the other variant's give other codes
+            other = oracle.sr_bytes(seed_sr, 1, variant)
+            assert not np.array_equal(other, oracle.sr_bytes(seed_sr, 0, variant))
+            assert not np.array_equal(oracle.sr_bytes(seed_sr, 0, 0), oracle.sr_bytes(seed_sr, 0, 1))
+
+
 # ------------------------------------------------------------------ the blockwise quantizer (Sec. 2.1, Sec. 4)
 
 def _rand_bits(rows, cols, seed, scale=1.0):
