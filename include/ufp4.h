@@ -237,6 +237,17 @@ int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t ld, const u
                   uint64_t seed_rht, double *dev_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The quantities of Sec. 3 from the 19 sums of ufp4_diagnose (both arrays in HOST memory; plain host arithmetic, no
+ * launch).  out (11 doubles):
+ *   [0] alpha = sum xq x' / sum x'^2, the operand projection of Eq. 3
+ *   [1] NMSE  = sum (xq - x')^2 / sum x'^2 (Sec. 3.3; Eq. 7's Delta SQNR is 10 log10 of the ratio of two of these)
+ *   [2] B_eff = exp(-sum_i p_i ln(p_i + 1e-12)) / 8, Eq. 6 over the K = 8 magnitude levels (zero included)
+ *   [3 + i] mean of (level_i - |x'| / s) over the elements on level i, Sec. 3.1's per-bin bias; NaN for an unused level
+ * [0] and [1] are NaN for an all-zero tensor.  Returns UFP4_ERR_NULL for a null pointer.
+ */
+int ufp4_diagnose_ratios(const double *sums, double *out);
+
+/*
  * ufp4_gemm without any device allocation by anyone (the paper has no counterpart to this entry point; it exists for
  * the library's users).  Some callers cannot provide the workspace ufp4_gemm's tensor-core path needs: a process
  * whose device memory has all been handed to a framework's pool, or code running at a point where calling cudaMalloc
@@ -244,7 +255,8 @@ int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t ld, const u
  * C[m][n] = sum_k a[m][k] * b[n][k] as ufp4_gemm(..., UFP4_PATH_TENSOR, ...) with its scratch (the decoded 8-bit
  * operands and the per-row reference scales) in a fixed device array that is part of the library image.
  *   - Limit: the scratch the shapes need, ufp4_gemm_workspace_bytes(A, B, UFP4_PATH_TENSOR), must not exceed
- *     ufp4_gemm_noalloc_max_scratch_bytes() (16 MiB: e.g. A and B of 2048 rows each at K = 4096); beyond it the call
+ *     ufp4_gemm_noalloc_max_scratch_bytes() (16 MiB: e.g. A of 2048 and B of 2040 rows at K = 4096 fit, 2048 and 2048 rows
+ *     do not, because the reference scales and the tile list share the array); beyond it the call
  *     returns UFP4_ERR_WORKSPACE and launches nothing.  Every GPU that loads the library holds those 16 MiB until exit.
  *   - Both operands must use UFP4_SCALE_POW2 (else UFP4_ERR_UNSUPPORTED).  C as in ufp4_gemm.
  *   - The first call on each device looks up the array's device address (that device must be current); make that first

@@ -63,6 +63,8 @@ def lib():
         L.orc_e4m3_encode.argtypes = [f32]
         L.orc_quantize.restype = i32
         L.orc_quantize.argtypes = [p, i64, i64, i64, i32, i32, i32, i32, i32, u64, u64, f32, p, p, p]
+        L.orc_quantize_window.restype = i32
+        L.orc_quantize_window.argtypes = [p, i64, i64, i64, i32, i32, i32, i32, i32, u64, u64, f32, p, p, p, i64, i64, i64]
         L.orc_dequantize.restype = None
         L.orc_dequantize.argtypes = [p, p, i64, i32, i32, f32, i64, i64, p]
         L.orc_gemm_f64.restype = None
@@ -174,7 +176,9 @@ def e4m3_encode(u: float) -> int:
 
 def quantize(x_bf16_bits: np.ndarray, axis: int, rht_block: int = 16, grid: int = GRID_INT4,
              rounding: int = ROUND_RTNE, scale_fmt: int = SCALE_FP32, seed_rht: int = 0, seed_sr: int = 0,
-             tensor_scale: float = 1.0, want_y: bool = False) -> QTensor:
+             tensor_scale: float = 1.0, want_y: bool = False, window=None) -> QTensor:
+    """window = (out_row0, kb0, full_nkb): x is a part of a larger tensor (see orc_quantize_window); only the SR draws
+    depend on it."""
     x = np.ascontiguousarray(x_bf16_bits)
     assert x.dtype == np.uint16 and x.ndim == 2
     rows, cols = x.shape
@@ -183,8 +187,10 @@ def quantize(x_bf16_bits: np.ndarray, axis: int, rht_block: int = 16, grid: int 
     codes = np.zeros((R, K // 2), dtype=np.uint8)
     scales = np.zeros((R, K // 16), dtype=np.uint8 if scale_fmt == SCALE_E4M3_TENSOR else np.float32)
     y = np.zeros((R, K), dtype=np.float32) if want_y else None
-    rc = lib().orc_quantize(_ptr(x), rows, cols, cols, axis, rht_block, grid, rounding, scale_fmt, seed_rht, seed_sr,
-                            tensor_scale, _ptr(codes), _ptr(scales), _ptr(y) if want_y else None)
+    out_row0, kb0, full_nkb = window if window is not None else (0, 0, K // 16)
+    rc = lib().orc_quantize_window(_ptr(x), rows, cols, cols, axis, rht_block, grid, rounding, scale_fmt, seed_rht, seed_sr,
+                                   tensor_scale, _ptr(codes), _ptr(scales), _ptr(y) if want_y else None,
+                                   out_row0, kb0, full_nkb)
     if rc != 0:
         raise ValueError("orc_quantize rejected its arguments")
     return QTensor(codes, scales, grid, scale_fmt, float(np.float32(tensor_scale)), y)

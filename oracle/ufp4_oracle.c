@@ -335,10 +335,30 @@ static void quantize_block(const float x[16], const orc_params *p, uint64_t bloc
  * scales is float[] for FP32 / POW2 and uint8_t[] for E4M3_TENSOR.  y_out (optional) receives the normalised
  * pre-rounding values in the output's [R][k] order.  Returns 0, or -1 on a bad shape / argument.
  */
+int orc_quantize_window(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int axis, int rht_block, int grid,
+                        int rounding, int scale_fmt, uint64_t seed_rht, uint64_t seed_sr, float tensor_scale,
+                        uint8_t *codes, void *scales, float *y_out, int64_t out_row0, int64_t kb0, int64_t full_nkb);
+
 int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int axis, int rht_block, int grid,
                  int rounding, int scale_fmt, uint64_t seed_rht, uint64_t seed_sr, float tensor_scale,
                  uint8_t *codes, void *scales, float *y_out) {
+    int64_t K = (axis == ORC_AXIS_ROW) ? cols : rows;
+    return orc_quantize_window(x, rows, cols, ld, axis, rht_block, grid, rounding, scale_fmt, seed_rht, seed_sr,
+                               tensor_scale, codes, scales, y_out, 0, 0, K / 16);
+}
+
+/*
+ * The same quantizer on a window of a larger tensor: x[rows][cols] is the part of the full tensor whose first output
+ * row (row for axis ROW, column for axis COL) is out_row0 and whose first 16-element block along the reduction axis is
+ * kb0, the full tensor having full_nkb blocks along that axis.  Only the SR draws depend on where a block sits in the
+ * full tensor (Philox counter = index of the block in the full variant's scales array); everything else is the
+ * window's own.  kb0 must be a multiple of the RHT block (and of 2 for 1x32 scale blocks) counted in 16-blocks.
+ */
+int orc_quantize_window(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int axis, int rht_block, int grid,
+                        int rounding, int scale_fmt, uint64_t seed_rht, uint64_t seed_sr, float tensor_scale,
+                        uint8_t *codes, void *scales, float *y_out, int64_t out_row0, int64_t kb0, int64_t full_nkb) {
     if (!x || !codes || !scales) return -1;
+    if (out_row0 < 0 || kb0 < 0 || full_nkb < 1) return -1;
     if (rht_block != 0 && rht_block != 16 && rht_block != 32 && rht_block != 64 && rht_block != 128) return -1;
     if (grid < 0 || grid > 4 || rounding < 0 || rounding > 1 || scale_fmt < 0 || scale_fmt > 3) return -1;
     int64_t R = (axis == ORC_AXIS_ROW) ? rows : cols; /* output rows   */
@@ -404,7 +424,7 @@ int orc_quantize(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, int 
             uint8_t nib[16];
             float sf;
             uint8_t sbyte;
-            uint64_t b = (uint64_t)(o * nkb + kb);
+            uint64_t b = (uint64_t)((out_row0 + o) * full_nkb + (kb0 + kb));
             quantize_block(xb, &p, b, (uint32_t)axis, nib, &sf, &sbyte, y_out ? y_out + (o * K + kb * 16) : NULL,
                            amax_shared);
             for (int j = 0; j < 8; ++j) codes[o * (K / 2) + kb * 8 + j] = (uint8_t)(nib[2 * j] | (nib[2 * j + 1] << 4));

@@ -26,7 +26,8 @@ LIB_PATH = os.path.join(_HERE, "libufp4.so")
 
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_rht_signs", "ufp4_qtensor_bytes", "ufp4_quantize",
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
-           "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes"]
+           "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes",
+           "ufp4_diagnose_ratios"]
 
 
 class _QTensorStruct(C.Structure):
@@ -80,6 +81,8 @@ def lib():
         L.ufp4_diagnose_workspace_bytes.argtypes = [i64, i64]
         L.ufp4_diagnose.restype = i32
         L.ufp4_diagnose.argtypes = [vp, i64, i64, i64, qp, i32, u64, vp, vp, sz, vp]
+        L.ufp4_diagnose_ratios.restype = i32
+        L.ufp4_diagnose_ratios.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double)]
         _lib = L
     return _lib
 
@@ -212,6 +215,14 @@ def diagnose(x: torch.Tensor, q_row: QTensor, rht_block: int = 16, seed_rht: int
     _check(lib().ufp4_diagnose(x.data_ptr(), rows, cols, x.stride(0), C.byref(s), rht_block, seed_rht, out.data_ptr(),
                                ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
     return out
+
+
+def diagnose_ratios(sums) -> list:
+    """ufp4_diagnose_ratios: [alpha, nmse, b_eff, bias of level 0..7] from the 19 sums (any host sequence of floats)."""
+    a = (C.c_double * 19)(*[float(v) for v in sums])
+    out = (C.c_double * 11)()
+    _check(lib().ufp4_diagnose_ratios(a, out))
+    return [float(v) for v in out]
 
 
 def gemm_workspace_bytes(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:

@@ -5,6 +5,8 @@
 // One pass over the BF16 matrix and its row variant: every thread walks 16-element blocks, recomputes x' = x H'_16 with
 // the quantizer's FP32 butterflies, and accumulates 19 sums; CTA partials go to the caller's workspace and a second,
 // single-CTA kernel adds them in a fixed order, so the result does not depend on scheduling.
+#include <math.h>
+
 #include "common.cuh"
 
 namespace ufp4 {
@@ -205,4 +207,23 @@ extern "C" int ufp4_diagnose(const void *x, int64_t rows, int64_t cols, int64_t 
     if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
     ufp4::diagnose_finish_kernel<<<1, 32 * ufp4::kDiagSums, 0, st>>>(P.partials, (int)ctas, dev_out);
     return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
+}
+
+// The ratios of Sec. 3 from the 19 sums above (host arithmetic on 19 numbers, no launch).
+extern "C" int ufp4_diagnose_ratios(const double *sums, double *out) {
+    if (!sums || !out) return UFP4_ERR_NULL;
+    const double sxx = sums[0];
+    const double qnan = NAN;
+    out[0] = sxx > 0.0 ? sums[2] / sxx : qnan;                       // alpha, Eq. 3
+    out[1] = sxx > 0.0 ? sums[1] / sxx : qnan;                       // NMSE, Sec. 3.3
+    double n = 0.0, ent = 0.0;
+    for (int i = 0; i < 8; ++i) n += sums[3 + i];
+    if (n > 0.0)
+        for (int i = 0; i < 8; ++i) {
+            const double p = sums[3 + i] / n;
+            ent -= p * log(p + 1e-12);                              // Eq. 6: natural logarithm, eps = 1e-12
+        }
+    out[2] = exp(ent) / 8.0;                                        // B_eff over K = 8 magnitude buckets
+    for (int i = 0; i < 8; ++i) out[3 + i] = sums[3 + i] > 0.0 ? sums[11 + i] / sums[3 + i] : qnan;
+    return UFP4_OK;
 }

@@ -255,7 +255,7 @@ gemm_promote_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // Per quant block: wait for its partial, copy this warp's 32 x 64 part out of tensor memory, hand the buffer
             // back to the MMA issuer at once (it runs up to kPBufs blocks ahead), then multiply the part in.
             for (int ks = 0; ok && ks < t.nks; ++ks) {
-                if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
                 const float *sA_s = reinterpret_cast<const float *>(smem + kPOffSA + stage * kPScaleStage);
                 const float *sB_s = reinterpret_cast<const float *>(smem + kPOffSB + stage * kPScaleStage);
 #pragma unroll 1
@@ -263,7 +263,7 @@ gemm_promote_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const float sa = sA_s[b * kTM + row];
                     const float2 sa2 = make_float2(sa, sa);
                     const float4 *sb4 = reinterpret_cast<const float4 *>(sB_s + b * kPN + cbase);
-                    if (!mbar_wait(pfull_bar + 8 * buf, bphase, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_warp(pfull_bar + 8 * buf, bphase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kPN + cbase);
                     uint32_t v0[32], v1[32];
@@ -458,13 +458,15 @@ int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, i
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
 
-    static int num_sms = 0;
-    if (!num_sms) {
-        int dev = 0;
-        UFP4_CUDA_OK(cudaGetDevice(&dev));
-        UFP4_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    static DeviceSetup slots[kMaxDevices];
+    const DeviceSetup *dev = nullptr;
+    const int rc_setup = device_setup(slots, [](int ordinal, DeviceSetup &d) -> int {
+        UFP4_CUDA_OK(cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, ordinal));
         UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_promote_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPSmem));
-    }
+        return UFP4_OK;
+    }, &dev);
+    if (rc_setup != UFP4_OK) return rc_setup;
+    const int num_sms = dev->num_sms;
     const int grid = (int)(total < num_sms ? total : num_sms);
     gemm_promote_kernel<<<grid, kPThreads, kPSmem, st>>>(tmA, tmB, tmSA, tmSB, tmC, P);
     return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;

@@ -359,18 +359,18 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                 // one buffer: wait until every epilogue thread has finished with the previous tile's values, write this
                 // tile's, and wait until all of them are there (bounded, abortable waits instead of bar.sync)
                 if (!first_tile) {
-                    if (!mbar_wait(rb_bar + 8, rb_read, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_warp(rb_bar + 8, rb_read, abort_flag)) { ok = false; break; }
                     rb_read ^= 1u;
                 }
                 first_tile = false;
                 refb_s[et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
                 mbar_arrive(rb_bar);
-                if (!mbar_wait(rb_bar, rb_written, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(rb_bar, rb_written, abort_flag)) { ok = false; break; }
                 rb_written ^= 1u;
             }
             const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s);
             if (has_k) {
-                if (!mbar_wait(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 acc_phase ^= 1u;
             }
@@ -579,23 +579,16 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
 
-    static int max_pairs = 0;
-    if (!max_pairs) {
-        int dev = 0, num_sms = 0;
-        UFP4_CUDA_OK(cudaGetDevice(&dev));
-        UFP4_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    static DeviceSetup slots[kMaxDevices];
+    const DeviceSetup *dev = nullptr;
+    const int rc_setup = device_setup(slots, [](int ordinal, DeviceSetup &d) -> int {
+        UFP4_CUDA_OK(cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, ordinal));
         UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSpSmem));
-        // how many CTA pairs can be resident at once (an SM whose neighbour is unavailable cannot host half a pair)
-        cudaLaunchConfig_t probe = {};
-        cudaLaunchAttribute pattr[1];
-        pattr[0].id = cudaLaunchAttributeClusterDimension;
-        pattr[0].val.clusterDim.x = 2; pattr[0].val.clusterDim.y = 1; pattr[0].val.clusterDim.z = 1;
-        probe.gridDim = dim3(2 * (num_sms / 2)); probe.blockDim = dim3(kSpThreads); probe.dynamicSmemBytes = kSpSmem;
-        probe.attrs = pattr; probe.numAttrs = 1;
-        int pairs = 0;
-        if (cudaOccupancyMaxActiveClusters(&pairs, gemm_split_kernel, &probe) != cudaSuccess || pairs < 1) pairs = num_sms / 2;
-        max_pairs = pairs;
-    }
+        d.max_pairs = resident_pairs(gemm_split_kernel, kSpThreads, kSpSmem, d.num_sms);
+        return UFP4_OK;
+    }, &dev);
+    if (rc_setup != UFP4_OK) return rc_setup;
+    const int max_pairs = dev->max_pairs;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;

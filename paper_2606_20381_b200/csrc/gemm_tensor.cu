@@ -344,18 +344,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // one buffer: wait until every epilogue thread has finished with the previous tile's values, write this
                 // tile's, and wait until all of them are there (bounded, abortable waits instead of bar.sync)
                 if (!first_tile) {
-                    if (!mbar_wait(rb_bar + 8, rb_read, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_warp(rb_bar + 8, rb_read, abort_flag)) { ok = false; break; }
                     rb_read ^= 1u;
                 }
                 first_tile = false;
                 refb_s[et] = n < P.N ? P.refB[t.b_row0 + n] : 0.0f;
                 mbar_arrive(rb_bar);
-                if (!mbar_wait(rb_bar, rb_written, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(rb_bar, rb_written, abort_flag)) { ok = false; break; }
                 rb_written ^= 1u;
             }
             const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s);
             if (t.nkb > 0) {
-                if (!mbar_wait(tfull_bar + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(tfull_bar + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
             }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTN;
@@ -575,24 +575,18 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
 
-    static int num_sms = 0, max_pairs = 0;
-    if (!num_sms) {
-        int dev = 0;
-        UFP4_CUDA_OK(cudaGetDevice(&dev));
-        UFP4_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    static DeviceSetup slots[kMaxDevices];
+    const DeviceSetup *dev = nullptr;
+    const int rc_setup = device_setup(slots, [](int ordinal, DeviceSetup &d) -> int {
+        UFP4_CUDA_OK(cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, ordinal));
         UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
         UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
-        // how many CTA pairs can be resident at once (an SM whose neighbour is unavailable cannot host half a pair)
-        cudaLaunchConfig_t probe = {};
-        cudaLaunchAttribute pattr[1];
-        pattr[0].id = cudaLaunchAttributeClusterDimension;
-        pattr[0].val.clusterDim.x = 2; pattr[0].val.clusterDim.y = 1; pattr[0].val.clusterDim.z = 1;
-        probe.gridDim = dim3(2 * (num_sms / 2)); probe.blockDim = dim3(kTcThreads); probe.dynamicSmemBytes = kTcSmem;
-        probe.attrs = pattr; probe.numAttrs = 1;
-        if (cudaOccupancyMaxActiveClusters(&max_pairs, gemm_tc_kernel<2>, &probe) != cudaSuccess || max_pairs < 1)
-            max_pairs = num_sms / 2;
-        if (getenv("UFP4_DEBUG")) fprintf(stderr, "[ufp4] SMs %d, resident CTA pairs %d\n", num_sms, max_pairs);
-    }
+        d.max_pairs = resident_pairs(gemm_tc_kernel<2>, kTcThreads, kTcSmem, d.num_sms);
+        if (getenv("UFP4_DEBUG")) fprintf(stderr, "[ufp4] device %d: SMs %d, resident CTA pairs %d\n", ordinal, d.num_sms, d.max_pairs);
+        return UFP4_OK;
+    }, &dev);
+    if (rc_setup != UFP4_OK) return rc_setup;
+    const int num_sms = dev->num_sms, max_pairs = dev->max_pairs;
     if (cg == 1) {
         const int grid = (int)(total < num_sms ? total : num_sms);
         gemm_tc_kernel<1><<<grid, kTcThreads, kTcSmem, st>>>(tmA, tmB, tmC, P);
@@ -619,8 +613,7 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
 constexpr size_t kNoAllocScratchBytes = (size_t)16 << 20;
 static __device__ __align__(256) uint8_t g_noalloc_scratch[kNoAllocScratchBytes];
 
-constexpr int kMaxDevices = 64;
-static void *g_noalloc_ptr[kMaxDevices] = {};
+static std::atomic<void *> g_noalloc_ptr[kMaxDevices];
 
 // Device address of the scratch array on the current device.  In host code the array's name is only a handle, not an
 // address a kernel could use, so the address is asked for once per device (with that device current) and cached.
@@ -628,12 +621,12 @@ static int noalloc_scratch(void **out) {
     int dev = 0;
     UFP4_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return UFP4_ERR_UNSUPPORTED;
-    if (!g_noalloc_ptr[dev]) {
-        void *p = nullptr;
-        UFP4_CUDA_OK(cudaGetSymbolAddress(&p, g_noalloc_scratch));
-        g_noalloc_ptr[dev] = p;
+    void *p = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
+        UFP4_CUDA_OK(cudaGetSymbolAddress(&p, g_noalloc_scratch));     // the same answer from every thread
+        g_noalloc_ptr[dev].store(p, std::memory_order_release);
     }
-    *out = g_noalloc_ptr[dev];
+    *out = p;
     return UFP4_OK;
 }
 

@@ -4,6 +4,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
+#include "../../include/ufp4.h"
 #include "ptx.cuh"
 
 namespace ufp4 {
@@ -181,6 +185,53 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uin
     asm volatile(
         "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// Once-per-device launcher set-up (kernel attributes, SM and resident-pair counts).  Kernel attributes belong to a
+// device's context, so a launcher keeps one slot per device ordinal; a slot is filled under its mutex and published
+// only after every step has succeeded (a failed set-up is retried by the next call).
+// ------------------------------------------------------------------------------------------------------------------
+constexpr int kMaxDevices = 64;
+
+struct DeviceSetup {
+    std::mutex mu;
+    std::atomic<int> ready{0};
+    int num_sms = 0, max_pairs = 0;
+};
+
+// Slot of the current device, filled by init(device ordinal, slot) on first use.  Returns a ufp4_status.
+template <class Init>
+inline int device_setup(DeviceSetup (&slots)[kMaxDevices], Init &&init, const DeviceSetup **out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return UFP4_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return UFP4_ERR_UNSUPPORTED;
+    DeviceSetup &d = slots[dev];
+    if (!d.ready.load(std::memory_order_acquire)) {
+        std::lock_guard<std::mutex> lock(d.mu);
+        if (!d.ready.load(std::memory_order_relaxed)) {
+            const int rc = init(dev, d);
+            if (rc != UFP4_OK) return rc;
+            d.ready.store(1, std::memory_order_release);
+        }
+    }
+    *out = &d;
+    return UFP4_OK;
+}
+
+// How many CTA pairs (clusters of 2) of `kernel` can be resident at once; an SM whose neighbour is unavailable cannot
+// host half a pair.
+template <class Kernel>
+inline int resident_pairs(Kernel kernel, int threads, int smem_bytes, int num_sms) {
+    cudaLaunchConfig_t probe = {};
+    cudaLaunchAttribute pattr[1];
+    pattr[0].id = cudaLaunchAttributeClusterDimension;
+    pattr[0].val.clusterDim.x = 2; pattr[0].val.clusterDim.y = 1; pattr[0].val.clusterDim.z = 1;
+    probe.gridDim = dim3(2 * (num_sms / 2)); probe.blockDim = dim3(threads); probe.dynamicSmemBytes = smem_bytes;
+    probe.attrs = pattr; probe.numAttrs = 1;
+    int pairs = 0;
+    if (cudaOccupancyMaxActiveClusters(&pairs, kernel, &probe) != cudaSuccess || pairs < 1) pairs = num_sms / 2;
+    return pairs;
 }
 
 }  // namespace ufp4

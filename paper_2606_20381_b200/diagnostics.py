@@ -1,10 +1,8 @@
-"""Measurement helpers around ufp4_diagnose (not part of the hot path): the Shrinkage-Bias diagnostic of Sec. 3.1,
-b_G = E[rho_G(t) - t] restricted to the bin of each level, the operand projection alpha of Eq. 3, the NMSE behind
-Eq. 7 and the effective bucket ratio of Eq. 6, for a tensor quantized by libufp4.  The sums come from the library's
-kernel; this module only turns them into ratios."""
+"""Measurement helpers around ufp4_diagnose (not part of the hot path): the Shrinkage-Bias diagnostic of Sec. 3.1, the
+operand projection alpha of Eq. 3, the NMSE behind Eq. 7 and the effective bucket ratio of Eq. 6, for a tensor
+quantized by libufp4.  Both the sums (a kernel) and the ratios (ufp4_diagnose_ratios) come from the library; this
+module only names the entries of what it returns."""
 from __future__ import annotations
-
-import math
 
 import torch
 
@@ -12,23 +10,14 @@ from . import binding as ufp4
 
 
 def tensor_diagnostics(x: torch.Tensor, q_row: ufp4.QTensor, rht_block: int, seed_rht: int) -> dict:
-    """alpha (Eq. 3), nmse (Sec. 3.3), b_eff (Eq. 6: natural log, eps = 1e-12, K = 8 magnitude buckets incl. zero),
-    count[8] and bias[8] (mean of level - t per magnitude level, NaN where a level is unused) of the row variant."""
+    """alpha, nmse, b_eff, count[8] and bias[8] (NaN where a level is unused) of the row variant q_row of x."""
     sums = ufp4.diagnose(x, q_row, rht_block, seed_rht).cpu()
-    count, bias_sum = sums[3:11], sums[11:19]
-    n = float(count.sum())
-    ent = -sum((float(c) / n) * math.log(float(c) / n + 1e-12) for c in count) if n > 0 else 0.0
-    sxx = float(sums[0])
-    return {"alpha": float(sums[2]) / sxx if sxx > 0 else float("nan"),
-            "nmse": float(sums[1]) / sxx if sxx > 0 else float("nan"),
-            "b_eff": math.exp(ent) / 8.0,
-            "count": count.to(torch.int64),
-            "bias": torch.where(count > 0, bias_sum / count.clamp_min(1), torch.full_like(bias_sum, float("nan"))),
-            "sums": sums}
+    r = ufp4.diagnose_ratios(sums.tolist())
+    return {"alpha": r[0], "nmse": r[1], "b_eff": r[2], "count": sums[3:11].to(torch.int64),
+            "bias": torch.tensor(r[3:11], dtype=torch.float64), "sums": sums}
 
 
 def per_bin_bias(x: torch.Tensor, q_row: ufp4.QTensor, rht_block: int, seed_rht: int):
-    """(count[8], mean of level - t per level) for the row variant q_row of the BF16 matrix x, t = |x'| / s in grid
-    units, x' the rotated input."""
+    """(count[8], mean of level - t per level) for the row variant q_row of the BF16 matrix x."""
     d = tensor_diagnostics(x, q_row, rht_block, seed_rht)
     return d["count"], d["bias"]

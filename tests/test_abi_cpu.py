@@ -120,3 +120,20 @@ def test_grouped_gemm_checks_offsets_on_the_host(lib):
     assert gg(C.byref(A), C.byref(B), 0x4000, 32, 0, 0, 1, None, C.cast(off, C.c_void_p), 2, 32, None, 0, None, None) == -1
     assert gg(C.byref(A), C.byref(_q(3 * 32, 64)), 0x4000, 32, 0, 0, 1, 0x8000, C.cast(off, C.c_void_p), 2, 32, None, 0,
               None, None) == -2
+
+
+def test_diagnose_ratios_is_host_arithmetic_and_matches_the_oracle(lib):
+    """ufp4_diagnose_ratios turns the 19 sums into alpha, NMSE, B_eff and the per-level bias on the host; the same
+    numbers from the oracle's own formulae."""
+    import numpy as np
+    sums = np.array([200.0, 3.0, 198.0, 10, 20, 30, 40, 0, 60, 70, 80, -2.5, 0.5, 0.25, -0.125, 0.0, 1.0, -1.0, 4.0])
+    got = ufp4.diagnose_ratios(sums.tolist())
+    want = oracle.diagnostics_from_sums(sums)
+    assert got[0] == pytest.approx(want["alpha"], rel=1e-15) and got[1] == pytest.approx(want["nmse"], rel=1e-15)
+    assert got[2] == pytest.approx(want["b_eff"], rel=1e-12)
+    assert np.isnan(got[3 + 4]) and np.isnan(want["bias"][4])
+    keep = [i for i in range(8) if i != 4]
+    assert np.allclose(np.array(got[3:])[keep], want["bias"][keep], rtol=1e-15)
+    zero = ufp4.diagnose_ratios([0.0] * 19)
+    assert np.isnan(zero[0]) and np.isnan(zero[1]) and zero[2] == pytest.approx(1.0 / 8.0)
+    assert lib.ufp4_diagnose_ratios(None, None) == -1

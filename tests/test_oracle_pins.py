@@ -390,6 +390,27 @@ def test_sr_draws_are_keyed_by_block_index_and_variant():
             assert not np.array_equal(oracle.sr_bytes(seed_sr, 0, 0), oracle.sr_bytes(seed_sr, 0, 1))
 
 
+def test_a_window_of_a_tensor_quantizes_like_that_part_of_the_whole():
+    """orc_quantize_window on a band (row band for the row layout, column band for the col layout, and a band along the
+    reduction axis) gives exactly the codes and scales the whole-tensor call gives there, SR draws included."""
+    rows, cols = 96, 160
+    bits = _rand_bits(rows, cols, 91)
+    for rounding in (ROUND_RTNE, ROUND_SR):
+        kw = dict(rht_block=16, grid=GRID_INT4, rounding=rounding, seed_rht=3, seed_sr=9)
+        full_r = oracle.quantize(bits, AXIS_ROW, **kw)
+        full_c = oracle.quantize(bits, AXIS_COL, **kw)
+        # rows 32..79, columns 48..127 of the tensor
+        r0, r1, c0, c1 = 32, 80, 48, 128
+        part = np.ascontiguousarray(bits[r0:r1, c0:c1])
+        w = oracle.quantize(part, AXIS_ROW, window=(r0, c0 // 16, cols // 16), **kw)
+        assert np.array_equal(w.codes, full_r.codes[r0:r1, c0 // 2:c1 // 2]) and np.array_equal(w.scales, full_r.scales[r0:r1, c0 // 16:c1 // 16])
+        w = oracle.quantize(part, AXIS_COL, window=(c0, r0 // 16, rows // 16), **kw)
+        assert np.array_equal(w.codes, full_c.codes[c0:c1, r0 // 2:r1 // 2]) and np.array_equal(w.scales, full_c.scales[c0:c1, r0 // 16:r1 // 16])
+        if rounding == ROUND_SR:     # and the window's place matters for SR
+            w0 = oracle.quantize(part, AXIS_ROW, **kw)
+            assert not np.array_equal(w0.codes, full_r.codes[r0:r1, c0 // 2:c1 // 2])
+
+
 # ------------------------------------------------------------------ the blockwise quantizer (Sec. 2.1, Sec. 4)
 
 def _rand_bits(rows, cols, seed, scale=1.0):
