@@ -173,7 +173,7 @@ int ufp4_selftest_division(int32_t *dev_mismatches, void *stream);
 size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path);
 
 /* GEMM paths (given a workspace of ufp4_gemm_workspace_bytes(A, B, path); without one AUTO falls back to EXACT).
- * AUTO:    TENSOR when both operands use POW2 scales, else SPLIT.
+ * AUTO:    TENSOR when both operands use POW2 scales, FP16 when both use E4M3 x tensor scales, else SPLIT.
  * EXACT:   CUDA-core kernel: integer block partials (dp4a) promoted with the two FP32 block scales, FP64 running sum;
  *          every grid and scale format, no workspace; the slow reference path.
  * TENSOR:  tcgen05 / TMEM kernel on 8-bit floating-point operands into which code x 2^e is folded exactly (POW2 scales
@@ -184,9 +184,16 @@ size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, i
  * SPLIT:   tcgen05 / TMEM kernel on FP16 operands: each dequantized value, relative to a per-row power-of-two
  *          reference, is split into two FP16 pieces (22 significant bits) and the product taken by three MMAs per K
  *          step; every grid and scale format (Table 1's FP32 scales), plain and grouped; blocks more than 2^26 below
- *          a row's largest scale are flushed and set UFP4_DEV_EXP_WINDOW. */
+ *          a row's largest scale are flushed and set UFP4_DEV_EXP_WINDOW.
+ * FP16:    the same kernels with one FP16 piece per value and one MMA per K step, for operands that BOTH carry
+ *          E4M3 block scales times a per-tensor FP32 scale (the two-level hierarchy Sec. 2.1's footnote names):
+ *          level x E4M3 value has at most 7 significant bits, so it is exact in FP16 without a row reference or an
+ *          exponent window, and the two tensor scales multiply the result once (they enter as RN(ts x E4M3 value) in
+ *          the definition: a relative difference of 2^-24 per operand, far inside the bound below).  Any other scale
+ *          format: UFP4_ERR_UNSUPPORTED. */
 typedef enum {
-    UFP4_PATH_AUTO = 0, UFP4_PATH_EXACT = 1, UFP4_PATH_TENSOR = 2, UFP4_PATH_PROMOTE = 3, UFP4_PATH_SPLIT = 4
+    UFP4_PATH_AUTO = 0, UFP4_PATH_EXACT = 1, UFP4_PATH_TENSOR = 2, UFP4_PATH_PROMOTE = 3, UFP4_PATH_SPLIT = 4,
+    UFP4_PATH_FP16 = 5
 } ufp4_gemm_path;
 
 /* Which path ufp4_gemm would take for these operands and this request (given a sufficient workspace), or a negative

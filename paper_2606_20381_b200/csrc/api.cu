@@ -29,7 +29,10 @@ int gemm_split_kernel_launches();
 bool gemm_split_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
 int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                       int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets, int num_groups,
-                      int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+                      int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream,
+                      bool single);
+size_t gemm_fp16_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
+bool gemm_fp16_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
 
 static int check_operand(const ufp4_qtensor *q) {
     if (!q || !q->codes || !q->scales) return UFP4_ERR_NULL;
@@ -46,7 +49,7 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                          int mode, int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                          int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                          void *stream) {
-    if (path < 0 || path > 4) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 5) return UFP4_ERR_ENUM;
     if (!C) return UFP4_ERR_NULL;
     if (ldc < N) return UFP4_ERR_SHAPE;
     if (!aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
@@ -61,6 +64,16 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                                       workspace, workspace_bytes, dev_status, stream);
         if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
     }
+    // FP16 (one piece): E4M3 x tensor scales on both operands
+    const bool fp16_ok = gemm_fp16_supported(A, B, M, N, K, mode);
+    if (path == UFP4_PATH_FP16 && !fp16_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_FP16 || (path == UFP4_PATH_AUTO && fp16_ok)) {
+        const size_t need = gemm_fp16_workspace_bytes(A->rows, B->rows, A->k);
+        if (workspace && workspace_bytes >= need)
+            return gemm_split_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
+                                     workspace, workspace_bytes, dev_status, stream, true);
+        if (path == UFP4_PATH_FP16) return UFP4_ERR_WORKSPACE;
+    }
     // SPLIT, or AUTO for scale formats the folded path cannot take
     const bool split_ok = gemm_split_supported(A, B, M, N, K, mode);
     if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
@@ -68,7 +81,7 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
         const size_t need = gemm_split_workspace_bytes(A->rows, B->rows, A->k);
         if (workspace && workspace_bytes >= need)
             return gemm_split_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
-                                     workspace, workspace_bytes, dev_status, stream);
+                                     workspace, workspace_bytes, dev_status, stream, false);
         if (path == UFP4_PATH_SPLIT) return UFP4_ERR_WORKSPACE;
     }
     // PROMOTE, or AUTO for what neither tensor-core operand form can take
@@ -117,7 +130,10 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     const bool pow2 = ufp4::is_pow2_fmt(A->scale_fmt) && ufp4::is_pow2_fmt(B->scale_fmt);
     if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
         return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
-    // AUTO takes SPLIT, and PROMOTE only where SPLIT does not apply: enough for either
+    const bool e4m3 = A->scale_fmt == UFP4_SCALE_E4M3_TENSOR && B->scale_fmt == UFP4_SCALE_E4M3_TENSOR;
+    if (path == UFP4_PATH_FP16) return e4m3 ? ufp4::gemm_fp16_workspace_bytes(A->rows, B->rows, A->k) : 0;
+    // AUTO takes FP16 for E4M3 x tensor scales, else SPLIT, and PROMOTE only where SPLIT does not apply: the two-piece
+    // workspace is enough for all of them
     const size_t split = ufp4::gemm_split_workspace_bytes(A->rows, B->rows, A->k);
     const size_t promote = ufp4::gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
     if (path == UFP4_PATH_SPLIT) return split;
@@ -130,18 +146,21 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (rc != UFP4_OK) return rc;
     rc = ufp4::check_operand(B);
     if (rc != UFP4_OK) return rc;
-    if (path < 0 || path > 4) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 5) return UFP4_ERR_ENUM;
     if (A->k != B->k) return UFP4_ERR_SHAPE;
     bool tensor_ok = ufp4::gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0);
     bool split_ok = ufp4::gemm_split_supported(A, B, A->rows, B->rows, A->k, 0);
+    bool fp16_ok = ufp4::gemm_fp16_supported(A, B, A->rows, B->rows, A->k, 0);
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_FP16 && !fp16_ok) return UFP4_ERR_UNSUPPORTED;
     int taken = path == UFP4_PATH_EXACT ? UFP4_PATH_EXACT
               : (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) ? UFP4_PATH_TENSOR
+              : (path == UFP4_PATH_FP16 || (path == UFP4_PATH_AUTO && fp16_ok)) ? UFP4_PATH_FP16
               : (path == UFP4_PATH_SPLIT || (path == UFP4_PATH_AUTO && split_ok)) ? UFP4_PATH_SPLIT : UFP4_PATH_PROMOTE;
     if (kernel_launches)
         *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : taken == UFP4_PATH_TENSOR ? ufp4::gemm_tensor_kernel_launches()
-                         : taken == UFP4_PATH_SPLIT ? ufp4::gemm_split_kernel_launches()
+                         : (taken == UFP4_PATH_SPLIT || taken == UFP4_PATH_FP16) ? ufp4::gemm_split_kernel_launches()
                                                     : ufp4::gemm_promote_kernel_launches();
     return taken;
 }

@@ -14,6 +14,12 @@
 //   2. gemm_split_kernel: the same warp-specialised, persistent CTA-pair design as the 8-bit kernel (TMA ring ->
 //      tcgen05.mma cta_group::2 kind::f16 -> tcgen05.ld epilogue -> TMA store), with four operand tiles per stage and
 //      the two accumulators filling tensor memory, so a tile's accumulators are read out before the next tile starts.
+//
+// One-piece variant (path FP16) for operands that both carry E4M3 block scales times a per-tensor FP32 scale (the
+// NVFP4-style two-level hierarchy of Sec. 2.1's footnote): level * E4M3 value has at most 3 + 4 significant bits and
+// lies in [2^-11, 3136], so it is exact in ONE FP16 number, needs no per-row reference and no exponent window, and the
+// per-tensor scales multiply the result once in the epilogue.  The same two kernels run with the lo pieces left out:
+// one MMA per K step, six operand stages instead of three and a double-buffered accumulator.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
@@ -31,6 +37,11 @@ constexpr int kSpTile = kTM * kTK;                    // bytes of one 128-row op
 constexpr int kSpStageBytes = 4 * kSpTile;            // hi_a, lo_a, hi_b (this CTA's half), lo_b (this CTA's half)
 constexpr int kSpStages = 3;
 constexpr int kSpRing = kSpStages * kSpStageBytes;
+// one-piece variant: hi_a and hi_b only, twice as many stages in the same ring
+constexpr int kSp1StageBytes = 2 * kSpTile;
+constexpr int kSp1Stages = 6;
+static_assert(kSp1Stages * kSp1StageBytes == kSpRing, "both variants use the same ring");
+constexpr int kSpMaxStages = 6;
 constexpr int kSpEpiWarps = 8;
 constexpr int kSpThreads = 64 + 32 * kSpEpiWarps;      // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-9: epilogue
 constexpr int kSpEpiBufBytes = 32 * 128;
@@ -65,6 +76,7 @@ struct SDecodeParams {
     int num_groups;
     int2 *mtiles;           // (first row, group) of every 256-row tile, group by group
     int32_t *dev_status;
+    int single;             // one-piece variant: both operands E4M3 x tensor scales; hi = level * E4M3 value, no lo
 };
 
 constexpr int kSDecodeThreads = 256;
@@ -115,7 +127,9 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
     // barrier is needed.  Four or eight warps per row: a thread scans the scales of its own blocks only and the warps
     // combine through shared memory.
     uint32_t smax = 0u;
-    if (TPR >= 128) {
+    if (P.single) {
+        // one-piece variant: no row reference, nothing to scan
+    } else if (TPR >= 128) {
         if (active) {
             int kb = t;
             for (; kb + 7 * TPR < nkb; kb += 8 * TPR) {
@@ -160,9 +174,16 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
     float n1, n2, r1, r2;
     pow2_factors(138 - fexp, &n1, &n2);                      // 2^(11 - e), e = fexp - 127
     pow2_factors(fexp - 138, &r1, &r2);
-    if (t == 0) O.ref[row] = smax == 0u ? 1.0f : __fmul_rn(r1, r2);
     const float unit = O.grid == UFP4_GRID_E1M2 ? 0.25f : (O.grid == UFP4_GRID_E2M1 ? 0.5f : 1.0f);
     n2 = __fmul_rn(n2, unit);
+    // one-piece variant: the operand is level * E4M3 value itself (exact in FP16); the tensor scale is the "reference"
+    const bool single = P.single != 0;
+    const float ts_mul = single ? 1.0f : ts;
+    if (single) {
+        n1 = 1.0f;
+        n2 = unit;
+    }
+    if (t == 0) O.ref[row] = single ? ts : (smax == 0u ? 1.0f : __fmul_rn(r1, r2));
 
     // Signed integer value of a nibble in its grid's unit (INT4: q, n >= 8 is n - 16; E1M2: +-(n & 7) quarters;
     // E2M1: +-{0,1,2,3,4,6,8,12} halves), offset by 16 so that it is a positive byte: a 16-entry table in four registers,
@@ -179,10 +200,10 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
     uint4 *lptr = reinterpret_cast<uint4 *>(O.lo + row * P.K);
 #pragma unroll 2
     for (int kb = t; kb < nkb; kb += TPR) {
-        const float s = split_scale_of(O, srow, kb, ts);
+        const float s = split_scale_of(O, srow, kb, ts_mul);
         uint2 cw = __ldg(cptr + kb);
         const float sn = __fmul_rn(__fmul_rn(s, n1), n2);           // normalised scale (with the level unit)
-        const bool keep = sn >= __uint_as_float((uint32_t)(kSpFlushExp + 127) << 23) * unit;
+        const bool keep = single ? true : sn >= __uint_as_float((uint32_t)(kSpFlushExp + 127) << 23) * unit;
         flushed |= (keep || s == 0.0f) ? 0u : (cw.x | cw.y);
         cw.x = keep ? cw.x : 0u;
         cw.y = keep ? cw.y : 0u;
@@ -212,9 +233,10 @@ __global__ void __launch_bounds__(kSDecodeThreads) decode_split_kernel(const SDe
         asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                      :: "l"(hptr + 2 * kb), "r"(hw[0]), "r"(hw[1]), "r"(hw[2]), "r"(hw[3]), "r"(hw[4]), "r"(hw[5]), "r"(hw[6]), "r"(hw[7])
                      : "memory");
-        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                     :: "l"(lptr + 2 * kb), "r"(lw[0]), "r"(lw[1]), "r"(lw[2]), "r"(lw[3]), "r"(lw[4]), "r"(lw[5]), "r"(lw[6]), "r"(lw[7])
-                     : "memory");
+        if (!single)
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                         :: "l"(lptr + 2 * kb), "r"(lw[0]), "r"(lw[1]), "r"(lw[2]), "r"(lw[3]), "r"(lw[4]), "r"(lw[5]), "r"(lw[6]), "r"(lw[7])
+                         : "memory");
     }
     if (flushed != 0u && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
 }
@@ -236,17 +258,21 @@ __device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t adesc,
 // [n0 + 128 r, +128) of both B pieces.  Accumulator 0 (columns 0..255 of tensor memory) takes hi_a hi_b, accumulator 1
 // (columns 256..511) takes hi_a lo_b + lo_a hi_b.  Tiles, reduction ranges and expert rows come from tile_info: plain
 // products, row-grouped products (256-row tiles laid out group by group) and reduction-grouped products alike.
+// SINGLE: the one-piece variant (hi pieces only, one MMA per K step, the two accumulators used in turn).
+template <bool SINGLE>
 __global__ void __launch_bounds__(kSpThreads, 1)
 gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constant__ CUtensorMap tmAl,
                   const __grid_constant__ CUtensorMap tmBh, const __grid_constant__ CUtensorMap tmBl,
                   const __grid_constant__ CUtensorMap tmC, const TcParams P) {
+    constexpr int kStages = SINGLE ? kSp1Stages : kSpStages;
+    constexpr int kStageBytes = SINGLE ? kSp1StageBytes : kSpStageBytes;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t base = smem_u32(smem);
     const uint32_t bars = base + kSpOffBars;
-    const uint32_t full_bar = bars, empty_bar = bars + 8 * kSpStages;
-    const uint32_t tfull_bar = bars + 16 * kSpStages, tempty_bar = tfull_bar + 8;
-    const uint32_t rb_bar = tempty_bar + 8;                 // two barriers: refB written / refB read by everyone
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kSpOffBars + 16 * kSpStages + 32);
+    const uint32_t full_bar = bars, empty_bar = bars + 8 * kSpMaxStages;
+    const uint32_t tfull_bar = bars + 16 * kSpMaxStages, tempty_bar = tfull_bar + 16;    // two of each (SINGLE uses both)
+    const uint32_t rb_bar = tempty_bar + 16;                // two barriers: refB written / refB read by everyone
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kSpOffBars + 16 * kSpMaxStages + 48);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -257,12 +283,14 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
     const int nks_all = (int)((P.K + kSpK - 1) / kSpK);      // K steps of a tile that reduces over all of K
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSpStages; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             mbar_init(full_bar + 8 * s, 2);                  // one arrive.expect_tx per CTA of the pair
             mbar_init(empty_bar + 8 * s, 1);
         }
-        mbar_init(tfull_bar, 1);
-        mbar_init(tempty_bar, 2 * kSpEpiWarps);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar + 8 * a, 1);
+            mbar_init(tempty_bar + 8 * a, 2 * kSpEpiWarps);
+        }
         mbar_init(rb_bar, 32 * kSpEpiWarps);
         mbar_init(rb_bar + 8, 32 * kSpEpiWarps);
         *abort_flag = (base & 1023u) ? 1u : 0u;             // the swizzled layouts below need the 1024-byte alignment
@@ -292,50 +320,62 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                 for (int ks = 0; ks < nks; ++ks) {
                     if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const int32_t kc = (ks0 + ks) * kSpK;
-                    const uint32_t fb = lead_full_bar + 8 * stage, dst = base + stage * kSpStageBytes;
-                    if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, kSpStageBytes);
-                    else mbar_expect_tx_cluster(fb, kSpStageBytes);
+                    const uint32_t fb = lead_full_bar + 8 * stage, dst = base + stage * kStageBytes;
+                    if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, kStageBytes);
+                    else mbar_expect_tx_cluster(fb, kStageBytes);
                     tma_load_2d_pair(dst, &tmAh, kc, m0, fb);
-                    tma_load_2d_pair(dst + kSpTile, &tmAl, kc, m0, fb);
-                    tma_load_2d_pair(dst + 2 * kSpTile, &tmBh, kc, n0, fb);
-                    tma_load_2d_pair(dst + 3 * kSpTile, &tmBl, kc, n0, fb);
-                    if (++stage == kSpStages) { stage = 0; phase ^= 1u; }
+                    if (SINGLE) {
+                        tma_load_2d_pair(dst + kSpTile, &tmBh, kc, n0, fb);
+                    } else {
+                        tma_load_2d_pair(dst + kSpTile, &tmAl, kc, m0, fb);
+                        tma_load_2d_pair(dst + 2 * kSpTile, &tmBh, kc, n0, fb);
+                        tma_load_2d_pair(dst + 3 * kSpTile, &tmBl, kc, n0, fb);
+                    }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             // ---------------- MMA issuer (rank 0 of the pair)
-            int stage = 0;
+            int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
                 const TileInfo t = tile_info<2>(P, tile, rank);
                 const int nks = P.mode == 2 ? 2 * t.nkb : nks_all;
                 if (nks == 0) continue;                       // empty group: the epilogue writes zeros
-                if (!mbar_wait(tempty_bar, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tempty_bar + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * kTN;
                 for (int ks = 0; ks < nks; ++ks) {
                     if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t st = base + stage * kSpStageBytes;
+                    const uint32_t st = base + stage * kStageBytes;
                     const uint64_t ah = umma_desc_sw128(st), al = umma_desc_sw128(st + kSpTile);
-                    const uint64_t bh = umma_desc_sw128(st + 2 * kSpTile), bl = umma_desc_sw128(st + 3 * kSpTile);
+                    const uint64_t bh = umma_desc_sw128(st + (SINGLE ? 1 : 2) * kSpTile), bl = umma_desc_sw128(st + 3 * kSpTile);
 #pragma unroll
                     for (int k = 0; k < kSpK / 16; ++k) {
                         // K = 16 FP16 elements = 32 bytes per instruction: +2 in the (address >> 4) field per step
                         const uint64_t o = (uint64_t)(2 * k);
                         const uint32_t first = (ks > 0 || k > 0) ? 1u : 0u;
-                        tc_mma_f16_pair(tmem_base, ah + o, bh + o, first);
-                        tc_mma_f16_pair(tmem_base + kTN, ah + o, bl + o, first);
-                        tc_mma_f16_pair(tmem_base + kTN, al + o, bh + o, 1u);
+                        tc_mma_f16_pair(d_tmem, ah + o, bh + o, first);
+                        if (!SINGLE) {
+                            tc_mma_f16_pair(tmem_base + kTN, ah + o, bl + o, first);
+                            tc_mma_f16_pair(tmem_base + kTN, al + o, bh + o, 1u);
+                        }
                     }
                     tc_commit<2>(empty_bar + 8 * stage);      // the stage is free (in both CTAs) once read
-                    if (++stage == kSpStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit<2>(tfull_bar);                      // both accumulators complete (in both CTAs)
-                acc_phase ^= 1u;
+                tc_commit<2>(tfull_bar + 8 * acc);            // the tile's accumulator(s) complete (in both CTAs)
+                if (SINGLE) {
+                    acc ^= 1;
+                    if (acc == 0) acc_phase ^= 1u;
+                } else {
+                    acc_phase ^= 1u;
+                }
             }
         }
     } else {
@@ -346,6 +386,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
         uint8_t *buf = smem + kSpOffEpi + (warp - 2) * kSpEpiBufBytes;
         float *refb_s = reinterpret_cast<float *>(smem + kSpOffRefB);
         uint32_t acc_phase = 0, rb_written = 0, rb_read = 0;
+        int acc = 0;
         bool first_tile = true;
         bool ok = true;
         for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
@@ -370,11 +411,20 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
             }
             const float4 *rb4 = reinterpret_cast<const float4 *>(refb_s);
             if (has_k) {
-                if (!mbar_wait_warp(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_warp(tfull_bar + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                acc_phase ^= 1u;
             }
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)acc * kTN;
+            const uint32_t lead_tempty = lead_tempty_bar + 8 * acc;
+            if (has_k) {
+                // which accumulator and barrier phase the next tile with a reduction uses
+                if (SINGLE) {
+                    acc ^= 1;
+                    if (acc == 0) acc_phase ^= 1u;
+                } else {
+                    acc_phase ^= 1u;
+                }
+            }
             const int32_t c_row = (int32_t)(m0 + q * 32), c_grp = (int32_t)(t.c_row0 / (P.M > 0 ? P.M : 1));
             uint32_t v0[32], v1[32];
 #pragma unroll
@@ -382,8 +432,12 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                 const int c = 4 * half + cc;
                 if (has_k) {
                     tc_ld32(taddr + (uint32_t)(c * 32), v0);
-                    tc_ld32(taddr + (uint32_t)(kTN + c * 32), v1);
+                    if (!SINGLE) tc_ld32(taddr + (uint32_t)(kTN + c * 32), v1);
                     tc_wait_ld();
+                    if (SINGLE) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v1[j] = 0u;
+                    }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v0[j] = v1[j] = 0u;
@@ -392,7 +446,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                     // every column of both accumulators has been read: hand them back to the MMA warp
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(lead_tempty_bar);
+                    if (lane == 0) mbar_arrive_cluster(lead_tempty);
                 }
                 const int64_t n_base = n0 + c * 32;
                 if (n_base >= P.N || c_row >= t.row_end) continue;   // warp-uniform: the box is clipped or not this tile's
@@ -487,6 +541,23 @@ size_t gemm_split_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K) {
 
 int gemm_split_kernel_launches() { return 2; }
 
+// one-piece variant (path FP16): the hi arrays only
+size_t gemm_fp16_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K) {
+    return sp_round_up((size_t)a_rows * K * 2, 256) + sp_round_up((size_t)b_rows * K * 2, 256) +
+           sp_round_up((size_t)a_rows * 4, 256) + sp_round_up((size_t)b_rows * 4, 256) +
+           sp_round_up((size_t)(a_rows / 128 + 2) * sizeof(int2), 256);
+}
+
+// level * E4M3 value is exact in FP16 (at most 7 significant bits, magnitudes in [2^-11, 3136]); the per-tensor FP32
+// scales multiply the result.  Other scale formats need the two-piece split.
+bool gemm_fp16_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode) {
+    (void)mode;
+    if (A->scale_fmt != UFP4_SCALE_E4M3_TENSOR || B->scale_fmt != UFP4_SCALE_E4M3_TENSOR) return false;
+    if (K % 16 != 0 || M < 1 || N < 1) return false;
+    if (A->rows > 0x3FFFFFFF || B->rows > 0x3FFFFFFF || K > 0x3FFFFFFF) return false;
+    return true;
+}
+
 bool gemm_split_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode) {
     (void)mode;
     if (K % 16 != 0 || M < 1 || N < 1) return false;
@@ -506,17 +577,21 @@ static bool sp_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// single: the one-piece variant (path FP16); the caller has checked gemm_fp16_supported.
 int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                       int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets, int num_groups,
-                      int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
+                      int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream,
+                      bool single) {
     if (!aligned_to(workspace, 256)) return UFP4_ERR_ALIGN;
-    if (workspace_bytes < gemm_split_workspace_bytes(A->rows, B->rows, K)) return UFP4_ERR_WORKSPACE;
+    if (workspace_bytes < (single ? gemm_fp16_workspace_bytes(A->rows, B->rows, K) : gemm_split_workspace_bytes(A->rows, B->rows, K)))
+        return UFP4_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     const size_t a_bytes = sp_round_up((size_t)A->rows * K * 2, 256), b_bytes = sp_round_up((size_t)B->rows * K * 2, 256);
-    __half *Ah = reinterpret_cast<__half *>(ws), *Al = reinterpret_cast<__half *>(ws + a_bytes);
-    __half *Bh = reinterpret_cast<__half *>(ws + 2 * a_bytes), *Bl = reinterpret_cast<__half *>(ws + 2 * a_bytes + b_bytes);
-    float *refA = reinterpret_cast<float *>(ws + 2 * a_bytes + 2 * b_bytes);
+    const size_t np = single ? 1 : 2;                                   // pieces per operand
+    __half *Ah = reinterpret_cast<__half *>(ws), *Al = single ? Ah : reinterpret_cast<__half *>(ws + a_bytes);
+    __half *Bh = reinterpret_cast<__half *>(ws + np * a_bytes), *Bl = single ? Bh : reinterpret_cast<__half *>(ws + 2 * a_bytes + b_bytes);
+    float *refA = reinterpret_cast<float *>(ws + np * a_bytes + np * b_bytes);
     float *refB = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(refA) + sp_round_up((size_t)A->rows * 4, 256));
     int2 *mtiles = reinterpret_cast<int2 *>(reinterpret_cast<uint8_t *>(refB) + sp_round_up((size_t)B->rows * 4, 256));
     // row-grouped product: 256-row tiles group by group (the decode launch lists them from the device offsets)
@@ -531,6 +606,7 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
                              B->ld_scales, B->rows, codebook_of(B->grid), B->scale_fmt, Bh, Bl, refB};
     D.K = K;
     D.dev_status = dev_status;
+    D.single = single ? 1 : 0;
     int tpr = 32;           // a warp per row up to 8 blocks per thread, more threads on longer rows
     while (tpr < kSDecodeThreads && (K >> 4) >= (int64_t)16 * tpr) tpr *= 2;
     const int64_t rows_per_cta = kSDecodeThreads / tpr;
@@ -583,8 +659,9 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
     const DeviceSetup *dev = nullptr;
     const int rc_setup = device_setup(slots, [](int ordinal, DeviceSetup &d) -> int {
         UFP4_CUDA_OK(cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, ordinal));
-        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSpSmem));
-        d.max_pairs = resident_pairs(gemm_split_kernel, kSpThreads, kSpSmem, d.num_sms);
+        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSpSmem));
+        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSpSmem));
+        d.max_pairs = resident_pairs(gemm_split_kernel<false>, kSpThreads, kSpSmem, d.num_sms);
         return UFP4_OK;
     }, &dev);
     if (rc_setup != UFP4_OK) return rc_setup;
@@ -599,8 +676,9 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_split_kernel, tmAh, tmAl, tmBh, tmBl, tmC, P) == cudaSuccess ? UFP4_OK
-                                                                                                        : UFP4_ERR_CUDA;
+    const cudaError_t err = single ? cudaLaunchKernelEx(&cfg, gemm_split_kernel<true>, tmAh, tmAl, tmBh, tmBl, tmC, P)
+                                   : cudaLaunchKernelEx(&cfg, gemm_split_kernel<false>, tmAh, tmAl, tmBh, tmBl, tmC, P);
+    return err == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 
 }  // namespace ufp4
