@@ -275,6 +275,18 @@ int ufp4_diagnose_ratios(const double *sums, double *out);
 int ufp4_gemm_noalloc(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16,
                       int32_t *dev_status, void *stream);
 
+/*
+ * Test hook for the failure path of the tensor-core kernels (TENSOR, SPLIT and FP16 paths; the paper has no
+ * counterpart).  Every wait of those kernels on a copy or on the tensor cores is bounded: after poll_limit polls (0 =
+ * the default, 2^24) the waiting role raises a flag in shared memory, the other roles see it in their own waits, the
+ * kernel returns normally (tensor memory released, cluster barriers met) and UFP4_DEV_WAIT_TIMEOUT is OR-ed into
+ * *dev_status.  With skip_loads = 1 the launches that follow issue no operand loads at all, so the first wait of the
+ * MMA-issuing thread runs out by construction, with no copy and no MMA in flight: that is how the tests exercise the
+ * path without faulting or hanging anything.  Process-wide until reset with (0, 0); C is left undefined by such a call.
+ * Returns UFP4_ERR_ENUM unless skip_loads is 0 or 1.
+ */
+int ufp4_debug_wait_injection(uint32_t poll_limit, int skip_loads);
+
 /* Size in bytes of the fixed scratch array behind ufp4_gemm_noalloc. */
 size_t ufp4_gemm_noalloc_max_scratch_bytes(void);
 

@@ -27,7 +27,7 @@ LIB_PATH = os.path.join(_HERE, "libufp4.so")
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_rht_signs", "ufp4_qtensor_bytes", "ufp4_quantize",
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
            "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes",
-           "ufp4_diagnose_ratios"]
+           "ufp4_diagnose_ratios", "ufp4_debug_wait_injection"]
 
 
 class _QTensorStruct(C.Structure):
@@ -81,6 +81,8 @@ def lib():
         L.ufp4_diagnose_workspace_bytes.argtypes = [i64, i64]
         L.ufp4_diagnose.restype = i32
         L.ufp4_diagnose.argtypes = [vp, i64, i64, i64, qp, i32, u64, vp, vp, sz, vp]
+        L.ufp4_debug_wait_injection.restype = i32
+        L.ufp4_debug_wait_injection.argtypes = [C.c_uint32, i32]
         L.ufp4_diagnose_ratios.restype = i32
         L.ufp4_diagnose_ratios.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double)]
         _lib = L
@@ -215,6 +217,11 @@ def diagnose(x: torch.Tensor, q_row: QTensor, rht_block: int = 16, seed_rht: int
     _check(lib().ufp4_diagnose(x.data_ptr(), rows, cols, x.stride(0), C.byref(s), rht_block, seed_rht, out.data_ptr(),
                                ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
     return out
+
+
+def debug_wait_injection(poll_limit: int = 0, skip_loads: bool = False):
+    """ufp4_debug_wait_injection: test hook, see include/ufp4.h.  Reset with debug_wait_injection()."""
+    _check(lib().ufp4_debug_wait_injection(poll_limit, 1 if skip_loads else 0))
 
 
 def diagnose_ratios(sums) -> list:

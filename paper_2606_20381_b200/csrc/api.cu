@@ -1,8 +1,16 @@
 // Host-side entry points of libufp4 that are not tied to one kernel file: version, status strings, size helpers and
 // the GEMM dispatch (argument validation, path selection).
+#include <atomic>
+
 #include "common.cuh"
 
 namespace ufp4 {
+// test hooks of the tensor-core launchers (ufp4_debug_wait_injection)
+static std::atomic<uint32_t> g_wait_limit{0};
+static std::atomic<int> g_skip_loads{0};
+uint32_t debug_wait_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
+int debug_skip_loads() { return g_skip_loads.load(std::memory_order_relaxed); }
+
 int gemm_exact_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                       int64_t M, int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n,
                       void *stream);
@@ -216,4 +224,11 @@ extern "C" int ufp4_gemm_noalloc(const ufp4_qtensor *A, const ufp4_qtensor *B, v
     if (A->k != B->k || ldc < B->rows) return UFP4_ERR_SHAPE;
     if (!ufp4::aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
     return ufp4::gemm_noalloc_launch(A, B, C, ldc, c_is_bf16, dev_status, stream);
+}
+
+extern "C" int ufp4_debug_wait_injection(uint32_t poll_limit, int skip_loads) {
+    if (skip_loads != 0 && skip_loads != 1) return UFP4_ERR_ENUM;
+    ufp4::g_wait_limit.store(poll_limit, std::memory_order_relaxed);
+    ufp4::g_skip_loads.store(skip_loads, std::memory_order_relaxed);
+    return UFP4_OK;
 }

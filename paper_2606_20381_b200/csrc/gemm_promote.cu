@@ -166,7 +166,7 @@ gemm_promote_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t bars = base + kPOffBars;
     const uint32_t full_bar = bars, empty_bar = bars + 32, pfull_bar = bars + 64, pempty_bar = bars + 96;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kPOffBars + 128);
-    volatile uint32_t *abort_flag = tmem_slot + 1;
+    volatile uint32_t *abort_flag = tmem_slot + 1;           // flag, poll limit
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -178,7 +178,8 @@ gemm_promote_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(pfull_bar + 8 * b, 1);
             mbar_init(pempty_bar + 8 * b, 8);
         }
-        *abort_flag = (base & 1023u) ? 1u : 0u;
+        abort_flag[0] = (base & 1023u) ? 1u : 0u;
+        abort_flag[1] = kWaitLimit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {

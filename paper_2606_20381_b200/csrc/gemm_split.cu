@@ -273,7 +273,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
     const uint32_t tfull_bar = bars + 16 * kSpMaxStages, tempty_bar = tfull_bar + 16;    // two of each (SINGLE uses both)
     const uint32_t rb_bar = tempty_bar + 16;                // two barriers: refB written / refB read by everyone
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kSpOffBars + 16 * kSpMaxStages + 48);
-    volatile uint32_t *abort_flag = tmem_slot + 1;
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kSpOffBars + 160);   // flag, poll limit
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = (int)cluster_cta_rank();
@@ -293,7 +293,8 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
         }
         mbar_init(rb_bar, 32 * kSpEpiWarps);
         mbar_init(rb_bar + 8, 32 * kSpEpiWarps);
-        *abort_flag = (base & 1023u) ? 1u : 0u;             // the swizzled layouts below need the 1024-byte alignment
+        abort_flag[0] = (base & 1023u) ? 1u : 0u;           // the swizzled layouts below need the 1024-byte alignment
+        abort_flag[1] = P.wait_limit ? P.wait_limit : kWaitLimit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -312,7 +313,7 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+            for (int tile = group_id; ok && !P.skip_loads && tile < P.total_tiles; tile += num_groups_launched) {
                 const TileInfo t = tile_info<2>(P, tile, rank);
                 const int32_t m0 = (int32_t)t.m0, n0 = (int32_t)(t.b_row0 + t.n0) + rank * (kTN / 2);
                 // tile_info counts the reduction in units of 128 elements; a K step here is 64
@@ -654,6 +655,8 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
+    P.wait_limit = debug_wait_limit();
+    P.skip_loads = debug_skip_loads();
 
     static DeviceSetup slots[kMaxDevices];
     const DeviceSetup *dev = nullptr;

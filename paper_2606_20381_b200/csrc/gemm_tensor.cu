@@ -227,7 +227,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t full_bar = bars, empty_bar = bars + 8 * kMaxStages;
     const uint32_t tfull_bar = bars + 16 * kMaxStages, tempty_bar = tfull_bar + 16;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kOffBars + 16 * kMaxStages + 32);
-    volatile uint32_t *abort_flag = tmem_slot + 1;
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kOffBars + 160);   // flag, poll limit
     const uint32_t rb_bar = bars + 16 * kMaxStages + 40;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -248,7 +248,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(tempty_bar + 8 * a, CG * kEpiWarps);
             mbar_init(rb_bar + 8 * a, 32 * kEpiWarps);
         }
-        *abort_flag = (base & 1023u) ? 1u : 0u;      // the swizzled layouts below need the 1024-byte alignment
+        abort_flag[0] = (base & 1023u) ? 1u : 0u;    // the swizzled layouts below need the 1024-byte alignment
+        abort_flag[1] = P.wait_limit ? P.wait_limit : kWaitLimit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -267,7 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+            for (int tile = group_id; ok && !P.skip_loads && tile < P.total_tiles; tile += num_groups_launched) {
                 const TileInfo t = tile_info<CG>(P, tile, rank);
                 for (int kb = 0; kb < t.nkb; ++kb) {
                     if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -574,6 +575,8 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
+    P.wait_limit = debug_wait_limit();
+    P.skip_loads = debug_skip_loads();
 
     static DeviceSetup slots[kMaxDevices];
     const DeviceSetup *dev = nullptr;

@@ -6,7 +6,7 @@
 
 namespace ufp4 {
 
-constexpr uint32_t kWaitLimit = 1u << 24;   // polls after which a bounded mbarrier wait gives up
+constexpr uint32_t kWaitLimit = 1u << 24;   // default number of polls after which a bounded mbarrier wait gives up
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -27,9 +27,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0u;
 }
 
-// Bounded wait: gives up after kWaitLimit polls or when another role has raised the abort flag.
+// Bounded wait: gives up after a number of polls or when another role has raised the abort flag.  abort_flag points at
+// two words of shared memory: [0] the flag, [1] the poll limit (kWaitLimit unless the launch asked for another).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint32_t limit = abort_flag[1];
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 64u) {
             if (*abort_flag) return false;

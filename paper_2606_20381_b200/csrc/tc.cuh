@@ -134,7 +134,15 @@ struct TcParams {
     // mode 1 on CTA pairs: the 256-row tiles are laid out group by group, so that a tile never straddles two groups;
     // entry i = (first row, group) of row-tile i (a group of 128 (mod 256) rows ends with a half-filled tile)
     const int2 *mtiles;
+    // test hooks (ufp4_debug_wait_injection; both 0 in normal use): the poll limit of every bounded wait, and a mode in
+    // which the TMA producer loads nothing, so that the MMA issuer's first wait runs out
+    uint32_t wait_limit;
+    int skip_loads;
 };
+
+// Process-wide test hooks behind ufp4_debug_wait_injection (defined in api.cu).
+uint32_t debug_wait_limit();
+int debug_skip_loads();
 
 struct TileInfo {
     int64_t m0, n0, b_row0, c_row0;
