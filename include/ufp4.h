@@ -212,6 +212,24 @@ int ufp4_gemm(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc
               void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 
 /*
+ * The same product with a quantizing epilogue (Sec. 5.5: "end-to-end training overhead still depends on full-system
+ * integration"): C = A B^T is rounded to BF16, as it would be stored for the next layer, and leaves the kernel already
+ * quantized the way ufp4_quantize(C, AXIS_BOTH, rht_block, UFP4_GRID_INT4, UFP4_ROUND_RTNE, scale_fmt, seed_rht) would
+ * quantize it: out_row [M][N] with its 1 x 16 blocks (and the RHT) along N, out_col [N][M] with them along M.  Either
+ * output may be NULL; C_bf16 [M][ldc] (optional, may be NULL) receives the BF16 product itself.  The FP32 product is
+ * never written: 1.5 B per element leave the kernel instead of 4.
+ *   A, B       POW2 scales (the tensor-core path); M and N multiples of 16
+ *   outputs    grid UFP4_GRID_INT4, scale_fmt UFP4_SCALE_FP32 or UFP4_SCALE_POW2 (the same for both); rht_block 16 or 0
+ *   workspace  ufp4_gemm_workspace_bytes(A, B, UFP4_PATH_TENSOR)
+ * For consumers that round to nearest (the next layer's X); SR consumers go through ufp4_quantize.  The codes are those
+ * of the BF16-rounded tensor-core result: where the exact product lies within the GEMM bound of a BF16 rounding
+ * boundary, the BF16 value, and with it codes of its block, can differ from those of the exactly rounded product.
+ */
+int ufp4_gemm_quantized(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C_bf16, int64_t ldc, int rht_block,
+                        uint64_t seed_rht, const ufp4_qtensor *out_row, const ufp4_qtensor *out_col, void *workspace,
+                        size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/*
  * MoE-grouped variant: one call for all experts.  offsets is a DEVICE int64 [num_groups+1] array of row offsets
  * (offsets[0] = 0, every offset a multiple of 128; padding rows must hold zero codes or zero scales), and
  * host_offsets the same values in HOST memory (the launch geometry is sized from them).

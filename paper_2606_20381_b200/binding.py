@@ -27,7 +27,7 @@ LIB_PATH = os.path.join(_HERE, "libufp4.so")
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_rht_signs", "ufp4_qtensor_bytes", "ufp4_quantize",
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
            "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes",
-           "ufp4_diagnose_ratios", "ufp4_debug_wait_injection"]
+           "ufp4_diagnose_ratios", "ufp4_debug_wait_injection", "ufp4_gemm_quantized"]
 
 
 class _QTensorStruct(C.Structure):
@@ -81,6 +81,8 @@ def lib():
         L.ufp4_diagnose_workspace_bytes.argtypes = [i64, i64]
         L.ufp4_diagnose.restype = i32
         L.ufp4_diagnose.argtypes = [vp, i64, i64, i64, qp, i32, u64, vp, vp, sz, vp]
+        L.ufp4_gemm_quantized.restype = i32
+        L.ufp4_gemm_quantized.argtypes = [qp, qp, vp, i64, i32, u64, qp, qp, vp, sz, vp, vp]
         L.ufp4_debug_wait_injection.restype = i32
         L.ufp4_debug_wait_injection.argtypes = [C.c_uint32, i32]
         L.ufp4_diagnose_ratios.restype = i32
@@ -217,6 +219,32 @@ def diagnose(x: torch.Tensor, q_row: QTensor, rht_block: int = 16, seed_rht: int
     _check(lib().ufp4_diagnose(x.data_ptr(), rows, cols, x.stride(0), C.byref(s), rht_block, seed_rht, out.data_ptr(),
                                ws.data_ptr(), ws.numel(), _stream_ptr(stream)))
     return out
+
+
+def gemm_quantized(A: QTensor, B: QTensor, rht_block: int = 16, seed_rht: int = 0, scale_fmt: int = SCALE_FP32,
+                   want_row: bool = True, want_col: bool = True, want_c: bool = False, out_row: QTensor | None = None,
+                   out_col: QTensor | None = None, out_c: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+                   dev_status: torch.Tensor | None = None, stream=None):
+    """ufp4_gemm_quantized: returns (row layout [M][N] or None, col layout [N][M] or None, BF16 C or None)."""
+    M, N = A.rows, B.rows
+    dev = A.codes.device
+    if want_row and out_row is None:
+        out_row = alloc_qtensor(M, N, GRID_INT4, scale_fmt, dev)
+    if want_col and out_col is None:
+        out_col = alloc_qtensor(N, M, GRID_INT4, scale_fmt, dev)
+    if want_c and out_c is None:
+        out_c = _alloc_out(M, N, True, dev)
+    if workspace is None:
+        workspace = torch.empty(max(16, gemm_workspace_bytes(A, B, PATH_TENSOR)), dtype=torch.uint8, device=dev)
+    sa, sb = A.struct(), B.struct()
+    sr = out_row.struct() if out_row is not None else None
+    sc = out_col.struct() if out_col is not None else None
+    _check(lib().ufp4_gemm_quantized(C.byref(sa), C.byref(sb), out_c.data_ptr() if out_c is not None else None,
+                                     out_c.stride(0) if out_c is not None else N, rht_block, seed_rht,
+                                     C.byref(sr) if sr is not None else None, C.byref(sc) if sc is not None else None,
+                                     workspace.data_ptr(), workspace.numel(),
+                                     dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
+    return out_row, out_col, out_c
 
 
 def debug_wait_injection(poll_limit: int = 0, skip_loads: bool = False):

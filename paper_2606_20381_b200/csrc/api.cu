@@ -20,10 +20,17 @@ int gemm_noalloc_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, i
                         int32_t *dev_status, void *stream);
 size_t gemm_noalloc_max_bytes();
 bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
+struct TcQOut {
+    uint8_t *row_codes, *col_codes;
+    float *row_scales, *col_scales;
+    int64_t row_ldc, row_lds, col_ldc, col_lds;
+    int rht, pow2;
+    uint32_t sign_mask;
+};
 int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                        int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                        int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
-                       void *stream);
+                       void *stream, const TcQOut *qout);
 
 size_t gemm_promote_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
 int gemm_promote_kernel_launches();
@@ -69,7 +76,7 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
         const size_t need = gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
         if (workspace && workspace_bytes >= need)
             return gemm_tensor_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
-                                      workspace, workspace_bytes, dev_status, stream);
+                                      workspace, workspace_bytes, dev_status, stream, nullptr);
         if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
     }
     // FP16 (one piece): E4M3 x tensor scales on both operands
@@ -231,4 +238,51 @@ extern "C" int ufp4_debug_wait_injection(uint32_t poll_limit, int skip_loads) {
     ufp4::g_wait_limit.store(poll_limit, std::memory_order_relaxed);
     ufp4::g_skip_loads.store(skip_loads, std::memory_order_relaxed);
     return UFP4_OK;
+}
+
+extern "C" int ufp4_gemm_quantized(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C_bf16, int64_t ldc, int rht_block,
+                                   uint64_t seed_rht, const ufp4_qtensor *out_row, const ufp4_qtensor *out_col,
+                                   void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream) {
+    int rc = ufp4::check_operand(A);
+    if (rc != UFP4_OK) return rc;
+    rc = ufp4::check_operand(B);
+    if (rc != UFP4_OK) return rc;
+    if (A->k != B->k) return UFP4_ERR_SHAPE;
+    if (rht_block != 0 && rht_block != 16) return UFP4_ERR_UNSUPPORTED;
+    if (!out_row && !out_col) return UFP4_ERR_NULL;
+    const int64_t M = A->rows, N = B->rows;
+    if (M % 16 != 0 || N % 16 != 0) return UFP4_ERR_SHAPE;
+    if (!ufp4::gemm_tensor_supported(A, B, M, N, A->k, 0)) return UFP4_ERR_UNSUPPORTED;
+    const ufp4_qtensor *any = out_row ? out_row : out_col;
+    const int fmt = any->scale_fmt;
+    if (fmt != UFP4_SCALE_FP32 && fmt != UFP4_SCALE_POW2) return UFP4_ERR_UNSUPPORTED;
+    for (int v = 0; v < 2; ++v) {
+        const ufp4_qtensor *q = v ? out_col : out_row;
+        if (!q) continue;
+        if (!q->codes || !q->scales) return UFP4_ERR_NULL;
+        if (q->grid != UFP4_GRID_INT4 || q->scale_fmt != fmt) return UFP4_ERR_UNSUPPORTED;
+        if (q->rows != (v ? N : M) || q->k != (v ? M : N)) return UFP4_ERR_SHAPE;
+        if (q->ld_codes_bytes < q->k / 2 || q->ld_codes_bytes % 16 != 0 || q->ld_scales < q->k / 16 ||
+            !ufp4::aligned_to(q->codes, 16) || !ufp4::aligned_to(q->scales, 4))
+            return UFP4_ERR_ALIGN;
+    }
+    if (C_bf16) {
+        if (ldc < N) return UFP4_ERR_SHAPE;
+        if (!ufp4::aligned_to(C_bf16, 16) || (ldc * 2) % 16 != 0) return UFP4_ERR_ALIGN;
+    }
+    if (!workspace || workspace_bytes < ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k)) return UFP4_ERR_WORKSPACE;
+    ufp4::TcQOut q = {};
+    if (out_row) {
+        q.row_codes = static_cast<uint8_t *>(out_row->codes); q.row_scales = static_cast<float *>(out_row->scales);
+        q.row_ldc = out_row->ld_codes_bytes; q.row_lds = out_row->ld_scales;
+    }
+    if (out_col) {
+        q.col_codes = static_cast<uint8_t *>(out_col->codes); q.col_scales = static_cast<float *>(out_col->scales);
+        q.col_ldc = out_col->ld_codes_bytes; q.col_lds = out_col->ld_scales;
+    }
+    q.rht = rht_block == 16;
+    q.pow2 = fmt == UFP4_SCALE_POW2;
+    q.sign_mask = ufp4_rht_sign_mask(seed_rht);
+    return ufp4::gemm_tensor_launch(A, B, C_bf16, C_bf16 ? ldc : N, 1, 0, M, N, A->k, nullptr, nullptr, 1, N, workspace,
+                                    workspace_bytes, dev_status, stream, &q);
 }

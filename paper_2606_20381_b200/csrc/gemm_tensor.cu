@@ -18,6 +18,7 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "quantize_core.cuh"
 #include "tc.cuh"
 
 namespace ufp4 {
@@ -214,7 +215,11 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const Decod
     if (flushed != 0u && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_EXP_WINDOW);
 }
 
-template <int CG>
+// QMODE 0: C leaves as FP32 or BF16.  QMODE 1 / 2 (quantizing epilogue, plain products only): C is rounded to BF16 and
+// quantized on the way out like ufp4_quantize would quantize it (uniform INT4 grid, RTNE, 1 x 16 blocks along N and
+// along M, 16-point RHT or none; FP32 scales for QMODE 1, power-of-two scales for QMODE 2); the BF16 C itself is
+// written only if P.C is given.
+template <int CG, int QMODE = 0>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const TcParams P) {
@@ -401,7 +406,89 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // the previous box must have been read out of the staging buffer by its TMA store
                 if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 __syncwarp();
-                if (P.c_is_bf16) {
+                if (QMODE != 0) {
+                    // ---- quantizing epilogue.  The BF16-rounded 32 x 32 box goes to the staging buffer in the BF16 store's
+                    // layout (64-byte rows, 16-byte piece j of row r at piece j ^ ((r >> 1) & 3)); the words a thread
+                    // builds for it, two adjacent columns each, are what the quantizer's row pass starts from.
+                    constexpr int QF = QMODE == 1 ? UFP4_SCALE_FP32 : UFP4_SCALE_POW2;
+                    uint32_t w[16];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float4 r0 = rb4[c * 8 + 2 * j], r1 = rb4[c * 8 + 2 * j + 1];
+                        const uint32_t *x = &v[cur][8 * j];
+                        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(x[0]) * ra * r0.x, __uint_as_float(x[1]) * ra * r0.y);
+                        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(x[2]) * ra * r0.z, __uint_as_float(x[3]) * ra * r0.w);
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(x[4]) * ra * r1.x, __uint_as_float(x[5]) * ra * r1.y);
+                        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(x[6]) * ra * r1.z, __uint_as_float(x[7]) * ra * r1.w);
+                        w[4 * j] = *reinterpret_cast<uint32_t *>(&h0); w[4 * j + 1] = *reinterpret_cast<uint32_t *>(&h1);
+                        w[4 * j + 2] = *reinterpret_cast<uint32_t *>(&h2); w[4 * j + 3] = *reinterpret_cast<uint32_t *>(&h3);
+                        *reinterpret_cast<uint4 *>(buf + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) =
+                            make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    }
+                    const QuantParams QP = {};                          // not read on the uniform-grid RTNE path
+                    bool nonfinite = false;
+                    if (P.q_row_codes) {
+                        // blocks along N: columns n_base .. +15 (words 0..7) and +16 .. +31 (words 8..15) of this thread's row
+                        float2 qv[16];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const uint32_t sl = P.q_rht ? P.q_sign_lo[j] : 0u, sh = P.q_rht ? P.q_sign_hi[j] : 0u;
+                            qv[2 * j] = make_float2(__uint_as_float(w[j] * 65536u + sl), __uint_as_float(w[8 + j] * 65536u + sl));
+                            qv[2 * j + 1] = make_float2(__uint_as_float((w[j] & 0xFFFF0000u) ^ sh), __uint_as_float((w[8 + j] & 0xFFFF0000u) ^ sh));
+                        }
+                        uint2 c0, c1;
+                        uint32_t s0, s1;
+                        if (P.q_rht) quantize_pair<GC_INT4, UFP4_ROUND_RTNE, QF, true>(qv, QP, 1.0f, 0, 0, 0u, &c0, &c1, &s0, &s1, &nonfinite);
+                        else quantize_pair<GC_INT4, UFP4_ROUND_RTNE, QF, false>(qv, QP, 1.0f, 0, 0, 0u, &c0, &c1, &s0, &s1, &nonfinite);
+                        if (m_own < t.row_end) {
+                            uint8_t *dst = P.q_row_codes + m_own * P.q_row_ldc + (n_base >> 1);
+                            float *sd = P.q_row_scales + m_own * P.q_row_lds + (n_base >> 4);
+                            if (n_base + 32 <= P.N) {
+                                *reinterpret_cast<uint4 *>(dst) = make_uint4(c0.x, c0.y, c1.x, c1.y);
+                                reinterpret_cast<uint32_t *>(sd)[0] = s0;
+                                reinterpret_cast<uint32_t *>(sd)[1] = s1;
+                            } else {                                   // N is a multiple of 16: the first block is inside
+                                *reinterpret_cast<uint2 *>(dst) = c0;
+                                *reinterpret_cast<uint32_t *>(sd) = s0;
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (P.q_col_codes) {
+                        // blocks along M: lane j takes column n_base + j of the staged box, rows 0..15 and 16..31
+                        const int64_t n_own = n_base + lane;
+                        float2 qv[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const uint32_t sc = P.q_rht ? P.q_sign[i] : 0u;
+                            const int r0i = i, r1i = 16 + i;
+                            const uint32_t e0 = *reinterpret_cast<const uint16_t *>(buf + r0i * 64 + (((lane >> 3) ^ ((r0i >> 1) & 3)) << 4) + ((lane & 7) << 1));
+                            const uint32_t e1 = *reinterpret_cast<const uint16_t *>(buf + r1i * 64 + (((lane >> 3) ^ ((r1i >> 1) & 3)) << 4) + ((lane & 7) << 1));
+                            qv[i] = make_float2(__uint_as_float(e0 * 65536u + sc), __uint_as_float(e1 * 65536u + sc));
+                        }
+                        uint2 c0, c1;
+                        uint32_t s0, s1;
+                        if (P.q_rht) quantize_pair<GC_INT4, UFP4_ROUND_RTNE, QF, true>(qv, QP, 1.0f, 0, 0, 0u, &c0, &c1, &s0, &s1, &nonfinite);
+                        else quantize_pair<GC_INT4, UFP4_ROUND_RTNE, QF, false>(qv, QP, 1.0f, 0, 0, 0u, &c0, &c1, &s0, &s1, &nonfinite);
+                        if (n_own < P.N) {
+                            uint8_t *dst = P.q_col_codes + n_own * P.q_col_ldc + (c_row >> 1);
+                            float *sd = P.q_col_scales + n_own * P.q_col_lds + (c_row >> 4);
+                            if (c_row + 32 <= t.row_end) {
+                                *reinterpret_cast<uint4 *>(dst) = make_uint4(c0.x, c0.y, c1.x, c1.y);
+                                reinterpret_cast<uint32_t *>(sd)[0] = s0;
+                                reinterpret_cast<uint32_t *>(sd)[1] = s1;
+                            } else {                                   // M is a multiple of 16: the first block is inside
+                                *reinterpret_cast<uint2 *>(dst) = c0;
+                                *reinterpret_cast<uint32_t *>(sd) = s0;
+                            }
+                        }
+                    }
+                    if (nonfinite && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_NONFINITE);
+                    if (!P.C) {                                        // no BF16 copy of C wanted: nothing for the TMA to store
+                        __syncwarp();
+                        continue;
+                    }
+                } else if (P.c_is_bf16) {
                     // 64-byte rows, 64B swizzle: 16-byte piece j of row r sits at piece j ^ ((r >> 1) & 3)
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -495,10 +582,11 @@ bool gemm_tensor_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t
     return true;
 }
 
+// qout (optional): the quantizing epilogue's outputs and settings; then C is BF16 or NULL and mode is 0.
 int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode,
                        int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                        int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
-                       void *stream) {
+                       void *stream, const TcQOut *qout) {
     if (!aligned_to(workspace, 256)) return UFP4_ERR_ALIGN;
     if (workspace_bytes < gemm_tensor_workspace_bytes(A->rows, B->rows, K)) return UFP4_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -547,8 +635,8 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
         return UFP4_ERR_CUDA;
 
     // C as [groups][rows][cols] so that the TMA store clips at the end of each group's rows and at N
-    CUtensorMap tmC;
-    {
+    CUtensorMap tmC = {};
+    if (C) {
         EncodeTiledFn fn = encode_tiled_fn();
         if (!fn) return UFP4_ERR_CUDA;
         const int64_t groups = mode == 2 ? num_groups : 1;
@@ -577,6 +665,18 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
     P.wait_limit = debug_wait_limit();
     P.skip_loads = debug_skip_loads();
+    int qmode = 0;
+    if (qout) {
+        qmode = qout->pow2 ? 2 : 1;
+        P.q_row_codes = qout->row_codes; P.q_row_scales = qout->row_scales; P.q_row_ldc = qout->row_ldc; P.q_row_lds = qout->row_lds;
+        P.q_col_codes = qout->col_codes; P.q_col_scales = qout->col_scales; P.q_col_ldc = qout->col_ldc; P.q_col_lds = qout->col_lds;
+        P.q_rht = qout->rht;
+        for (int j = 0; j < 8; ++j) {
+            P.q_sign_lo[j] = ((qout->sign_mask >> (2 * j)) & 1u) << 31;
+            P.q_sign_hi[j] = ((qout->sign_mask >> (2 * j + 1)) & 1u) << 31;
+        }
+        for (int i = 0; i < 16; ++i) P.q_sign[i] = ((qout->sign_mask >> i) & 1u) << 31;
+    }
 
     static DeviceSetup slots[kMaxDevices];
     const DeviceSetup *dev = nullptr;
@@ -584,6 +684,8 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
         UFP4_CUDA_OK(cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, ordinal));
         UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
         UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
+        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
+        UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem));
         d.max_pairs = resident_pairs(gemm_tc_kernel<2>, kTcThreads, kTcSmem, d.num_sms);
         if (getenv("UFP4_DEBUG")) fprintf(stderr, "[ufp4] device %d: SMs %d, resident CTA pairs %d\n", ordinal, d.num_sms, d.max_pairs);
         return UFP4_OK;
@@ -605,7 +707,11 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, tmA, tmB, tmC, P) == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
+    cudaError_t err;
+    if (qmode == 1) err = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 1>, tmA, tmB, tmC, P);
+    else if (qmode == 2) err = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 2>, tmA, tmB, tmC, P);
+    else err = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, tmA, tmB, tmC, P);
+    return err == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------------------------
@@ -641,7 +747,7 @@ int gemm_noalloc_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, i
     int rc = noalloc_scratch(&scratch);
     if (rc != UFP4_OK) return rc;
     return gemm_tensor_launch(A, B, C, ldc, c_is_bf16, 0, A->rows, B->rows, A->k, nullptr, nullptr, 1, B->rows, scratch,
-                              kNoAllocScratchBytes, dev_status, stream);
+                              kNoAllocScratchBytes, dev_status, stream, nullptr);
 }
 
 size_t gemm_noalloc_max_bytes() { return kNoAllocScratchBytes; }

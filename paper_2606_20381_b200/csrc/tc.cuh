@@ -134,10 +134,26 @@ struct TcParams {
     // mode 1 on CTA pairs: the 256-row tiles are laid out group by group, so that a tile never straddles two groups;
     // entry i = (first row, group) of row-tile i (a group of 128 (mod 256) rows ends with a half-filled tile)
     const int2 *mtiles;
+    // quantizing epilogue (ufp4_gemm_quantized): the product, rounded to BF16, leaves as the next consumer's quantized
+    // operand: blocks along N ("row" layout [M][N]) and / or blocks along M ("col" layout, stored [N][M])
+    uint8_t *q_row_codes, *q_col_codes;
+    float *q_row_scales, *q_col_scales;
+    int64_t q_row_ldc, q_row_lds, q_col_ldc, q_col_lds;
+    uint32_t q_sign_lo[8], q_sign_hi[8], q_sign[16];   // bit 31 set where eps of element 2j / 2j+1 / i of a block is -1
+    int q_rht;                                          // 16-point RHT before quantizing (else none)
     // test hooks (ufp4_debug_wait_injection; both 0 in normal use): the poll limit of every bounded wait, and a mode in
     // which the TMA producer loads nothing, so that the MMA issuer's first wait runs out
     uint32_t wait_limit;
     int skip_loads;
+};
+
+// Host-side description of the quantizing epilogue's outputs (gemm_tensor_launch).
+struct TcQOut {
+    uint8_t *row_codes, *col_codes;
+    float *row_scales, *col_scales;
+    int64_t row_ldc, row_lds, col_ldc, col_lds;
+    int rht, pow2;
+    uint32_t sign_mask;
 };
 
 // Process-wide test hooks behind ufp4_debug_wait_injection (defined in api.cu).
