@@ -302,68 +302,19 @@ gemm_promote_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int c = 0; c < 2; ++c) {
                 const int64_t n_base = t.n0 + cbase + 32 * c;
                 if (n_base >= P.N || c_row >= P.M) continue;
-                if (n_base + 32 > P.N && P.n_unaligned) {
-                    if (m_own < P.M) {
+                float x[32];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (n_base + j < P.N) {
-                                const float2 a2 = acc[16 * c + (j >> 1)];
-                                const float val = (j & 1) ? a2.y : a2.x;
-                                const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
-                                if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(val);
-                                else static_cast<float *>(P.C)[idx] = val;
-                            }
-                        }
-                    }
-                    continue;
+                for (int j = 0; j < 16; ++j) {
+                    x[2 * j] = acc[16 * c + j].x;
+                    x[2 * j + 1] = acc[16 * c + j].y;
                 }
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                __syncwarp();
-                if (P.c_is_bf16) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint32_t h[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const float2 a2 = acc[16 * c + 4 * j + u];
-                            __nv_bfloat162 hh = __floats2bfloat162_rn(a2.x, a2.y);
-                            h[u] = *reinterpret_cast<uint32_t *>(&hh);
-                        }
-                        *reinterpret_cast<uint4 *>(buf_st + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float2 a0 = acc[16 * c + 2 * j], a1 = acc[16 * c + 2 * j + 1];
-                        *reinterpret_cast<float4 *>(buf_st + lane * 128 + ((j ^ (lane & 7)) << 4)) = make_float4(a0.x, a0.y, a1.x, a1.y);
-                    }
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) {
-                    asm volatile(
-                        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
-                        ::"l"(&tmC), "r"((int32_t)n_base), "r"(c_row), "r"(c_grp), "r"(smem_u32(buf_st)) : "memory");
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                }
+                if (n_base + 32 > P.N && P.n_unaligned) epi_store_box_plain(P, x, t.c_row0 + m_own, n_base, m_own < P.M);
+                else epi_store_box_tma(P, &tmC, buf_st, lane, x, (int32_t)n_base, c_row, c_grp);
             }
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        __syncwarp();
+        epi_store_drain(lane);
     }
-
-    // ---------------- teardown
-    tc_fence_before();
-    __syncthreads();
-    if (*abort_flag) {
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-        if (threadIdx.x == 0 && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_WAIT_TIMEOUT);
-    }
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc<1>(tmem_base, kPBufs * kPN);
-    }
+    tc_teardown<1>(abort_flag, P.dev_status, tmem_base, kPBufs * kPN, warp);
 }
 
 // ------------------------------------------------------------------------------------------------------------------

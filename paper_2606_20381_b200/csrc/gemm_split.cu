@@ -451,80 +451,23 @@ gemm_split_kernel(const __grid_constant__ CUtensorMap tmAh, const __grid_constan
                 }
                 const int64_t n_base = n0 + c * 32;
                 if (n_base >= P.N || c_row >= t.row_end) continue;   // warp-uniform: the box is clipped or not this tile's
-                if (n_base + 32 > P.N && P.n_unaligned) {
-                    // The TMA clips in 16-byte units: a last chunk whose valid part does not end on a 16-byte boundary
-                    // is written with plain predicated stores so that nothing right of column N is touched.
-                    if (m_own < t.row_end) {
-                        for (int j = 0; j < 32 && n_base + j < P.N; ++j) {
-                            const float sum = __fmaf_rn(__uint_as_float(v1[j]), 1.0f / kSpLoScale, __uint_as_float(v0[j]));
-                            const float val = sum * ra * refb_s[c * 32 + j];
-                            const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
-                            if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(val);
-                            else static_cast<float *>(P.C)[idx] = val;
-                        }
-                    }
-                    continue;
-                }
-                // the previous box must have been read out of the staging buffer by its TMA store
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                __syncwarp();
                 float x[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    x[j] = __fmaf_rn(__uint_as_float(v1[j]), 1.0f / kSpLoScale, __uint_as_float(v0[j])) * ra;
-                if (P.c_is_bf16) {
-                    // 64-byte rows, 64B swizzle: 16-byte piece j of row r sits at piece j ^ ((r >> 1) & 3)
+                for (int j = 0; j < 8; ++j) {
+                    const float4 r = rb4[c * 8 + j];
+                    const float rr[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float4 r0 = rb4[c * 8 + 2 * j], r1 = rb4[c * 8 + 2 * j + 1];
-                        const float *y = &x[8 * j];
-                        __nv_bfloat162 h0 = __floats2bfloat162_rn(y[0] * r0.x, y[1] * r0.y);
-                        __nv_bfloat162 h1 = __floats2bfloat162_rn(y[2] * r0.z, y[3] * r0.w);
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(y[4] * r1.x, y[5] * r1.y);
-                        __nv_bfloat162 h3 = __floats2bfloat162_rn(y[6] * r1.z, y[7] * r1.w);
-                        *reinterpret_cast<uint4 *>(buf + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) =
-                            make_uint4(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1),
-                                       *reinterpret_cast<uint32_t *>(&h2), *reinterpret_cast<uint32_t *>(&h3));
-                    }
-                } else {
-                    // 128-byte rows, 128B swizzle: 16-byte piece j of row r sits at piece j ^ (r & 7)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float4 r = rb4[c * 8 + j];
-                        const float *y = &x[4 * j];
-                        *reinterpret_cast<float4 *>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                            make_float4(y[0] * r.x, y[1] * r.y, y[2] * r.z, y[3] * r.w);
-                    }
+                    for (int u = 0; u < 4; ++u)
+                        x[4 * j + u] = __fmaf_rn(__uint_as_float(v1[4 * j + u]), 1.0f / kSpLoScale, __uint_as_float(v0[4 * j + u])) * ra * rr[u];
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) {
-                    asm volatile(
-                        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
-                        ::"l"(&tmC), "r"((int32_t)n_base), "r"(c_row), "r"(c_grp), "r"(smem_u32(buf)) : "memory");
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                }
+                if (n_base + 32 > P.N && P.n_unaligned) epi_store_box_plain(P, x, t.c_row0 + m_own, n_base, m_own < t.row_end);
+                else epi_store_box_tma(P, &tmC, buf, lane, x, (int32_t)n_base, c_row, c_grp);
             }
             mbar_arrive(rb_bar + 8);                           // this thread has finished with the tile's refB values
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all C boxes written
-        __syncwarp();
+        epi_store_drain(lane);
     }
-
-    // ---------------- teardown
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                                    // neither CTA leaves while the other may still signal its barriers
-    if (*abort_flag) {
-        // a bounded wait gave up: let any copy still in flight land before shared memory is released
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-        if (threadIdx.x == 0 && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_WAIT_TIMEOUT);
-    }
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc<2>(tmem_base, 512);
-    }
+    tc_teardown<2>(abort_flag, P.dev_status, tmem_base, 512, warp);
 }
 
 // ------------------------------------------------------------------------------------------------------------------

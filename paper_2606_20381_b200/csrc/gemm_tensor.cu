@@ -391,22 +391,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int64_t n_base = t.n0 + c * 32;
                 if (n_base >= P.N || c_row >= t.row_end) continue;     // warp-uniform: the whole box is clipped or not this tile's
                 if (n_base + 32 > P.N && P.n_unaligned) {
-                    // The TMA clips in 16-byte units: a last chunk whose valid part does not end on a 16-byte boundary
-                    // is written with plain predicated stores so that nothing right of column N is touched.
-                    if (m_own < t.row_end) {
-                        for (int j = 0; j < 32 && n_base + j < P.N; ++j) {
-                            const float val = __uint_as_float(v[cur][j]) * ra * refb_s[c * 32 + j];
-                            const int64_t idx = (t.c_row0 + m_own) * P.ldc + n_base + j;
-                            if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(val);
-                            else static_cast<float *>(P.C)[idx] = val;
-                        }
-                    }
+                    float x[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(v[cur][j]) * ra * refb_s[c * 32 + j];
+                    epi_store_box_plain(P, x, t.c_row0 + m_own, n_base, m_own < t.row_end);
                     continue;
                 }
-                // the previous box must have been read out of the staging buffer by its TMA store
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                __syncwarp();
                 if (QMODE != 0) {
+                    // the previous box must have been read out of the staging buffer by its TMA store
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    __syncwarp();
                     // ---- quantizing epilogue.  The BF16-rounded 32 x 32 box goes to the staging buffer in the BF16 store's
                     // layout (64-byte rows, 16-byte piece j of row r at piece j ^ ((r >> 1) & 3)); the words a thread
                     // builds for it, two adjacent columns each, are what the quantizer's row pass starts from.
@@ -488,31 +482,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         __syncwarp();
                         continue;
                     }
-                } else if (P.c_is_bf16) {
-                    // 64-byte rows, 64B swizzle: 16-byte piece j of row r sits at piece j ^ ((r >> 1) & 3)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float4 r0 = rb4[c * 8 + 2 * j], r1 = rb4[c * 8 + 2 * j + 1];
-                        const uint32_t *x = &v[cur][8 * j];
-                        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(x[0]) * ra * r0.x, __uint_as_float(x[1]) * ra * r0.y);
-                        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(x[2]) * ra * r0.z, __uint_as_float(x[3]) * ra * r0.w);
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(x[4]) * ra * r1.x, __uint_as_float(x[5]) * ra * r1.y);
-                        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(x[6]) * ra * r1.z, __uint_as_float(x[7]) * ra * r1.w);
-                        *reinterpret_cast<uint4 *>(buf + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) =
-                            make_uint4(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1),
-                                       *reinterpret_cast<uint32_t *>(&h2), *reinterpret_cast<uint32_t *>(&h3));
-                    }
                 } else {
-                    // 128-byte rows, 128B swizzle: 16-byte piece j of row r sits at piece j ^ (r & 7)
+                    float x[32];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const float4 r = rb4[c * 8 + j];
-                        const uint32_t *x = &v[cur][4 * j];
-                        *reinterpret_cast<float4 *>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                            make_float4(__uint_as_float(x[0]) * ra * r.x, __uint_as_float(x[1]) * ra * r.y,
-                                        __uint_as_float(x[2]) * ra * r.z, __uint_as_float(x[3]) * ra * r.w);
+                        x[4 * j] = __uint_as_float(v[cur][4 * j]) * ra * r.x;
+                        x[4 * j + 1] = __uint_as_float(v[cur][4 * j + 1]) * ra * r.y;
+                        x[4 * j + 2] = __uint_as_float(v[cur][4 * j + 2]) * ra * r.z;
+                        x[4 * j + 3] = __uint_as_float(v[cur][4 * j + 3]) * ra * r.w;
                     }
+                    epi_store_box_tma(P, &tmC, buf, lane, x, (int32_t)n_base, c_row, c_grp);
+                    continue;
                 }
+                // QMODE with a BF16 copy of C: the box is already staged
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) {
@@ -528,24 +511,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (acc == 0) acc_phase ^= 1u;
             }
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all C boxes written
-        __syncwarp();
+        epi_store_drain(lane);
     }
-
-    // ---------------- teardown
-    tc_fence_before();
-    __syncthreads();
-    if (CG == 2) cluster_sync_all();                   // neither CTA leaves while the other may still signal its barriers
-    if (*abort_flag) {
-        // a bounded wait gave up: let any copy still in flight land before shared memory is released
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-        if (threadIdx.x == 0 && P.dev_status) atomicOr(P.dev_status, (int)UFP4_DEV_WAIT_TIMEOUT);
-    }
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc<CG>(tmem_base, kTmemCols);
-    }
+    tc_teardown<CG>(abort_flag, P.dev_status, tmem_base, kTmemCols, warp);
 }
 
 // ------------------------------------------------------------------------------------------------------------------

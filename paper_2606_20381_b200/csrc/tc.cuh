@@ -1,6 +1,7 @@
 // tcgen05 / tensor-memory wrappers and the tile bookkeeping shared by the tensor-core GEMM kernels (sm_100a).
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -201,6 +202,85 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams &P, int tile, int r
         t.c_row0 = (int64_t)g * P.M;
     }
     return t;
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// Epilogue and teardown pieces shared by the tensor-core kernels.  A warp owns a 32 x 32 box of C: lane = row of the box,
+// x[j] = that row's finished value in column j.
+// ------------------------------------------------------------------------------------------------------------------
+
+// A box on the right edge whose valid part does not end on a 16-byte boundary (the TMA clips in 16-byte units): plain
+// predicated stores, so that nothing right of column N is touched.  row = the lane's row of C (group offset included).
+__device__ __forceinline__ void epi_store_box_plain(const TcParams &P, const float (&x)[32], int64_t row, int64_t n_base,
+                                                    bool row_valid) {
+    if (!row_valid) return;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        if (n_base + j < P.N) {
+            const int64_t idx = row * P.ldc + n_base + j;
+            if (P.c_is_bf16) static_cast<__nv_bfloat16 *>(P.C)[idx] = __float2bfloat16_rn(x[j]);
+            else static_cast<float *>(P.C)[idx] = x[j];
+        }
+    }
+}
+
+// The box through the warp's staging buffer (4 KB) and one TMA store, which clips rows and columns outside C.  FP32: 128-byte
+// rows in the 128B swizzle pattern (16-byte piece j of row r at piece j ^ (r & 7)); BF16: 64-byte rows in the 64B pattern
+// (piece j at j ^ ((r >> 1) & 3)).  The previous box must have been read out of the buffer by its store first.
+__device__ __forceinline__ void epi_store_box_tma(const TcParams &P, const CUtensorMap *tmC, uint8_t *buf, int lane,
+                                                  const float (&x)[32], int32_t n_base, int32_t c_row, int32_t c_grp) {
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    __syncwarp();
+    if (P.c_is_bf16) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t h[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                __nv_bfloat162 hh = __floats2bfloat162_rn(x[8 * j + 2 * u], x[8 * j + 2 * u + 1]);
+                h[u] = *reinterpret_cast<uint32_t *>(&hh);
+            }
+            *reinterpret_cast<uint4 *>(buf + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) = make_uint4(h[0], h[1], h[2], h[3]);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<float4 *>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) {
+        asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                     ::"l"(tmC), "r"(n_base), "r"(c_row), "r"(c_grp), "r"(smem_u32(buf)) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+}
+
+// End of an epilogue warp's work: every box it handed to the TMA has been written.
+__device__ __forceinline__ void epi_store_drain(int lane) {
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
+}
+
+// Common exit of a tensor-core kernel: all roles meet (CTA, and the pair for CG = 2, so that neither CTA leaves while the
+// other may still signal its barriers); if a bounded wait gave up, copies still in flight get time to land before shared
+// memory is released and UFP4_DEV_WAIT_TIMEOUT is reported; the allocating warp (warp 1) returns the tensor memory.
+template <int CG>
+__device__ __forceinline__ void tc_teardown(volatile uint32_t *abort_flag, int32_t *dev_status, uint32_t tmem_base,
+                                            uint32_t tmem_cols, int warp) {
+    tc_fence_before();
+    __syncthreads();
+    if (CG == 2) cluster_sync_all();
+    if (*abort_flag) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0 && dev_status) atomicOr(dev_status, (int)UFP4_DEV_WAIT_TIMEOUT);
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc<CG>(tmem_base, tmem_cols);
+    }
 }
 
 
