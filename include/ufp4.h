@@ -305,6 +305,16 @@ int ufp4_gemm_noalloc(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
  */
 int ufp4_debug_wait_injection(uint32_t poll_limit, int skip_loads);
 
+/*
+ * Measurement aid (the paper has no counterpart; not on the hot path): cycles a scheduler of this GPU needs per group of
+ * warp instructions, for the instruction kinds the quantizer is made of: host_cycles (HOST, 8 doubles) receives
+ *   [0] add.rn.f32x2   [1] two add.rn.f32   [2] lop3   [3] mad.lo.u32   [4] f32x2 add + lop3   [5] f32x2 add + mad
+ *   [6] f32x2 add + two lop3   [7] two add.rn.f32 + lop3
+ * measured with one CTA of 1024 threads per SM on independent chains.  dev_scratch: device memory, 256-byte aligned, at
+ * least (SM count x 4096 + 256) bytes.  Synchronizes the stream.
+ */
+int ufp4_probe_issue_rates(void *dev_scratch, size_t scratch_bytes, double *host_cycles, void *stream);
+
 /* Size in bytes of the fixed scratch array behind ufp4_gemm_noalloc. */
 size_t ufp4_gemm_noalloc_max_scratch_bytes(void);
 

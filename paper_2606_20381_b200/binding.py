@@ -27,7 +27,8 @@ LIB_PATH = os.path.join(_HERE, "libufp4.so")
 EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_rht_signs", "ufp4_qtensor_bytes", "ufp4_quantize",
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
            "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes",
-           "ufp4_diagnose_ratios", "ufp4_debug_wait_injection", "ufp4_gemm_quantized"]
+           "ufp4_diagnose_ratios", "ufp4_debug_wait_injection", "ufp4_gemm_quantized",
+           "ufp4_probe_issue_rates"]
 
 
 class _QTensorStruct(C.Structure):
@@ -83,6 +84,8 @@ def lib():
         L.ufp4_diagnose.argtypes = [vp, i64, i64, i64, qp, i32, u64, vp, vp, sz, vp]
         L.ufp4_gemm_quantized.restype = i32
         L.ufp4_gemm_quantized.argtypes = [qp, qp, vp, i64, i32, u64, qp, qp, vp, sz, vp, vp]
+        L.ufp4_probe_issue_rates.restype = i32
+        L.ufp4_probe_issue_rates.argtypes = [vp, sz, C.POINTER(C.c_double), vp]
         L.ufp4_debug_wait_injection.restype = i32
         L.ufp4_debug_wait_injection.argtypes = [C.c_uint32, i32]
         L.ufp4_diagnose_ratios.restype = i32
@@ -245,6 +248,16 @@ def gemm_quantized(A: QTensor, B: QTensor, rht_block: int = 16, seed_rht: int = 
                                      workspace.data_ptr(), workspace.numel(),
                                      dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
     return out_row, out_col, out_c
+
+
+def probe_issue_rates(stream=None) -> dict:
+    """ufp4_probe_issue_rates: cycles per scheduler and group of warp instructions (see include/ufp4.h)."""
+    scratch = torch.empty(256 * 4096 + 256, dtype=torch.uint8, device="cuda")
+    out = (C.c_double * 8)()
+    _check(lib().ufp4_probe_issue_rates(scratch.data_ptr(), scratch.numel(), out, _stream_ptr(stream)))
+    names = ["add.f32x2", "add.f32, add.f32", "lop3", "mad.lo", "add.f32x2, lop3", "add.f32x2, mad.lo",
+             "add.f32x2, lop3, lop3", "add.f32, add.f32, lop3"]
+    return {n: float(v) for n, v in zip(names, out)}
 
 
 def debug_wait_injection(poll_limit: int = 0, skip_loads: bool = False):
