@@ -46,6 +46,12 @@ int gemm_split_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int
                       int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets, int num_groups,
                       int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream,
                       bool single);
+size_t gemm_mx_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
+int gemm_mx_kernel_launches();
+bool gemm_mx_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
+int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode, int64_t M,
+                   int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n, void *workspace,
+                   size_t workspace_bytes, int32_t *dev_status, void *stream);
 size_t gemm_fp16_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
 bool gemm_fp16_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
 
@@ -64,7 +70,7 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                          int mode, int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                          int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                          void *stream) {
-    if (path < 0 || path > 5) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 6) return UFP4_ERR_ENUM;
     if (!C) return UFP4_ERR_NULL;
     if (ldc < N) return UFP4_ERR_SHAPE;
     if (!aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
@@ -72,6 +78,17 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_EXACT)
         return gemm_exact_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, stream);
+    // MX (hardware block scaling): on request, and what AUTO takes when both operands carry 1 x 32 E8M0 scales
+    const bool mx_ok = gemm_mx_supported(A, B, M, N, K, mode);
+    const bool mx_auto = mx_ok && A->scale_fmt == UFP4_SCALE_E8M0_B32 && B->scale_fmt == UFP4_SCALE_E8M0_B32;
+    if (path == UFP4_PATH_MX && !mx_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_MX || (path == UFP4_PATH_AUTO && mx_auto)) {
+        const size_t need = gemm_mx_workspace_bytes(A->rows, B->rows, A->k);
+        if (workspace && workspace_bytes >= need)
+            return gemm_mx_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, workspace,
+                                  workspace_bytes, dev_status, stream);
+        if (path == UFP4_PATH_MX) return UFP4_ERR_WORKSPACE;
+    }
     if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) {
         const size_t need = gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
         if (workspace && workspace_bytes >= need)
@@ -143,8 +160,13 @@ extern "C" int ufp4_qtensor_bytes(int64_t rows, int64_t k, int scale_fmt, size_t
 extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path) {
     if (!A || !B || path == UFP4_PATH_EXACT) return 0;
     const bool pow2 = ufp4::is_pow2_fmt(A->scale_fmt) && ufp4::is_pow2_fmt(B->scale_fmt);
-    if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
-        return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
+    if (path == UFP4_PATH_MX) return pow2 ? ufp4::gemm_mx_workspace_bytes(A->rows, B->rows, A->k) : 0;
+    if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2)) {
+        // AUTO takes MX for two 1 x 32 tensors (plain and reduction-grouped products) and TENSOR otherwise: enough for both
+        const size_t t = pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
+        const size_t m = (path == UFP4_PATH_AUTO && pow2) ? ufp4::gemm_mx_workspace_bytes(A->rows, B->rows, A->k) : 0;
+        return t > m ? t : m;
+    }
     const bool e4m3 = A->scale_fmt == UFP4_SCALE_E4M3_TENSOR && B->scale_fmt == UFP4_SCALE_E4M3_TENSOR;
     if (path == UFP4_PATH_FP16) return e4m3 ? ufp4::gemm_fp16_workspace_bytes(A->rows, B->rows, A->k) : 0;
     // AUTO takes FP16 for E4M3 x tensor scales, else SPLIT, and PROMOTE only where SPLIT does not apply: the two-piece
@@ -161,8 +183,11 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (rc != UFP4_OK) return rc;
     rc = ufp4::check_operand(B);
     if (rc != UFP4_OK) return rc;
-    if (path < 0 || path > 5) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 6) return UFP4_ERR_ENUM;
     if (A->k != B->k) return UFP4_ERR_SHAPE;
+    bool mx_ok = ufp4::gemm_mx_supported(A, B, A->rows, B->rows, A->k, 0);
+    bool mx_auto = mx_ok && A->scale_fmt == UFP4_SCALE_E8M0_B32 && B->scale_fmt == UFP4_SCALE_E8M0_B32;
+    if (path == UFP4_PATH_MX && !mx_ok) return UFP4_ERR_UNSUPPORTED;
     bool tensor_ok = ufp4::gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0);
     bool split_ok = ufp4::gemm_split_supported(A, B, A->rows, B->rows, A->k, 0);
     bool fp16_ok = ufp4::gemm_fp16_supported(A, B, A->rows, B->rows, A->k, 0);
@@ -170,11 +195,13 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_FP16 && !fp16_ok) return UFP4_ERR_UNSUPPORTED;
     int taken = path == UFP4_PATH_EXACT ? UFP4_PATH_EXACT
+              : (path == UFP4_PATH_MX || (path == UFP4_PATH_AUTO && mx_auto)) ? UFP4_PATH_MX
               : (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) ? UFP4_PATH_TENSOR
               : (path == UFP4_PATH_FP16 || (path == UFP4_PATH_AUTO && fp16_ok)) ? UFP4_PATH_FP16
               : (path == UFP4_PATH_SPLIT || (path == UFP4_PATH_AUTO && split_ok)) ? UFP4_PATH_SPLIT : UFP4_PATH_PROMOTE;
     if (kernel_launches)
-        *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : taken == UFP4_PATH_TENSOR ? ufp4::gemm_tensor_kernel_launches()
+        *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : taken == UFP4_PATH_MX ? ufp4::gemm_mx_kernel_launches()
+                         : taken == UFP4_PATH_TENSOR ? ufp4::gemm_tensor_kernel_launches()
                          : (taken == UFP4_PATH_SPLIT || taken == UFP4_PATH_FP16) ? ufp4::gemm_split_kernel_launches()
                                                     : ufp4::gemm_promote_kernel_launches();
     return taken;
