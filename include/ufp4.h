@@ -173,8 +173,8 @@ int ufp4_selftest_division(int32_t *dev_mismatches, void *stream);
 size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path);
 
 /* GEMM paths (given a workspace of ufp4_gemm_workspace_bytes(A, B, path); without one AUTO falls back to EXACT).
- * AUTO:    MX when both operands use 1 x 32 E8M0 scales (plain and reduction-grouped products), TENSOR when both use
- *          power-of-two scales otherwise, FP16 when both use E4M3 x tensor scales, else SPLIT.
+ * AUTO:    TENSOR when both operands use power-of-two scales (1 x 16 or 1 x 32), FP16 when both use E4M3 x tensor
+ *          scales, else SPLIT.
  * EXACT:   CUDA-core kernel: integer block partials (dp4a) promoted with the two FP32 block scales, FP64 running sum;
  *          every grid and scale format, no workspace; the slow reference path.
  * TENSOR:  tcgen05 / TMEM kernel on 8-bit floating-point operands into which code x 2^e is folded exactly (POW2 scales
@@ -198,7 +198,9 @@ size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, i
  *          operands must carry power-of-two scales: UFP4_SCALE_E8M0_B32 is exact by construction (nothing is ever
  *          flushed), UFP4_SCALE_POW2 folds the gap between the two 16-blocks of a 32-group into the elements (a block
  *          more than 2^14 below its neighbour is flushed and sets UFP4_DEV_EXP_WINDOW).  Plain and reduction-grouped
- *          products; a row-grouped product returns UFP4_ERR_UNSUPPORTED (AUTO takes TENSOR for it). */
+ *          products; a row-grouped product returns UFP4_ERR_UNSUPPORTED.  On request only: on the same operands TENSOR
+ *          is the faster path (its accumulators are double-buffered and it copies no scales inside the main loop), so
+ *          MX is the choice for rows whose block exponents spread beyond TENSOR's window. */
 typedef enum {
     UFP4_PATH_AUTO = 0, UFP4_PATH_EXACT = 1, UFP4_PATH_TENSOR = 2, UFP4_PATH_PROMOTE = 3, UFP4_PATH_SPLIT = 4,
     UFP4_PATH_FP16 = 5, UFP4_PATH_MX = 6

@@ -78,16 +78,12 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_EXACT)
         return gemm_exact_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, stream);
-    // MX (hardware block scaling): on request, and what AUTO takes when both operands carry 1 x 32 E8M0 scales
-    const bool mx_ok = gemm_mx_supported(A, B, M, N, K, mode);
-    const bool mx_auto = mx_ok && A->scale_fmt == UFP4_SCALE_E8M0_B32 && B->scale_fmt == UFP4_SCALE_E8M0_B32;
-    if (path == UFP4_PATH_MX && !mx_ok) return UFP4_ERR_UNSUPPORTED;
-    if (path == UFP4_PATH_MX || (path == UFP4_PATH_AUTO && mx_auto)) {
-        const size_t need = gemm_mx_workspace_bytes(A->rows, B->rows, A->k);
-        if (workspace && workspace_bytes >= need)
-            return gemm_mx_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, workspace,
-                                  workspace_bytes, dev_status, stream);
-        if (path == UFP4_PATH_MX) return UFP4_ERR_WORKSPACE;
+    // MX (hardware block scaling): on request only; the folded path is the faster one on the same operands
+    if (path == UFP4_PATH_MX) {
+        if (!gemm_mx_supported(A, B, M, N, K, mode)) return UFP4_ERR_UNSUPPORTED;
+        if (!workspace || workspace_bytes < gemm_mx_workspace_bytes(A->rows, B->rows, A->k)) return UFP4_ERR_WORKSPACE;
+        return gemm_mx_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, num_groups, group_n, workspace,
+                              workspace_bytes, dev_status, stream);
     }
     if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) {
         const size_t need = gemm_tensor_workspace_bytes(A->rows, B->rows, A->k);
@@ -161,12 +157,8 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     if (!A || !B || path == UFP4_PATH_EXACT) return 0;
     const bool pow2 = ufp4::is_pow2_fmt(A->scale_fmt) && ufp4::is_pow2_fmt(B->scale_fmt);
     if (path == UFP4_PATH_MX) return pow2 ? ufp4::gemm_mx_workspace_bytes(A->rows, B->rows, A->k) : 0;
-    if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2)) {
-        // AUTO takes MX for two 1 x 32 tensors (plain and reduction-grouped products) and TENSOR otherwise: enough for both
-        const size_t t = pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
-        const size_t m = (path == UFP4_PATH_AUTO && pow2) ? ufp4::gemm_mx_workspace_bytes(A->rows, B->rows, A->k) : 0;
-        return t > m ? t : m;
-    }
+    if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
+        return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
     const bool e4m3 = A->scale_fmt == UFP4_SCALE_E4M3_TENSOR && B->scale_fmt == UFP4_SCALE_E4M3_TENSOR;
     if (path == UFP4_PATH_FP16) return e4m3 ? ufp4::gemm_fp16_workspace_bytes(A->rows, B->rows, A->k) : 0;
     // AUTO takes FP16 for E4M3 x tensor scales, else SPLIT, and PROMOTE only where SPLIT does not apply: the two-piece
@@ -185,9 +177,7 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (rc != UFP4_OK) return rc;
     if (path < 0 || path > 6) return UFP4_ERR_ENUM;
     if (A->k != B->k) return UFP4_ERR_SHAPE;
-    bool mx_ok = ufp4::gemm_mx_supported(A, B, A->rows, B->rows, A->k, 0);
-    bool mx_auto = mx_ok && A->scale_fmt == UFP4_SCALE_E8M0_B32 && B->scale_fmt == UFP4_SCALE_E8M0_B32;
-    if (path == UFP4_PATH_MX && !mx_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_MX && !ufp4::gemm_mx_supported(A, B, A->rows, B->rows, A->k, 0)) return UFP4_ERR_UNSUPPORTED;
     bool tensor_ok = ufp4::gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0);
     bool split_ok = ufp4::gemm_split_supported(A, B, A->rows, B->rows, A->k, 0);
     bool fp16_ok = ufp4::gemm_fp16_supported(A, B, A->rows, B->rows, A->k, 0);
@@ -195,7 +185,7 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_FP16 && !fp16_ok) return UFP4_ERR_UNSUPPORTED;
     int taken = path == UFP4_PATH_EXACT ? UFP4_PATH_EXACT
-              : (path == UFP4_PATH_MX || (path == UFP4_PATH_AUTO && mx_auto)) ? UFP4_PATH_MX
+              : path == UFP4_PATH_MX ? UFP4_PATH_MX
               : (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) ? UFP4_PATH_TENSOR
               : (path == UFP4_PATH_FP16 || (path == UFP4_PATH_AUTO && fp16_ok)) ? UFP4_PATH_FP16
               : (path == UFP4_PATH_SPLIT || (path == UFP4_PATH_AUTO && split_ok)) ? UFP4_PATH_SPLIT : UFP4_PATH_PROMOTE;

@@ -9,13 +9,18 @@
 // a block is flushed (and UFP4_DEV_EXP_WINDOW set) only if it lies more than 2^14 below the other half of its own
 // 32-group, which a 1 x 32 tensor cannot do by construction.  Two kernels:
 //   1. decode_mx_kernel: packed nibbles + scales -> E5M2 bytes [rows][K] and UE8M0 scale bytes in the 512-byte units the
-//      tensor core's scale copy takes: unit (row tile of 128, K step of 128) holds byte (row r, 32-group j) at
-//      (r % 32) * 16 + (r / 32) * 4 + j.
-//   2. gemm_mx_kernel: persistent, warp-specialised, one CTA per 128 x 256 tile: TMA brings operand tiles and scale units
-//      into a 3-stage ring; the MMA thread copies a stage's scales to tensor memory (tcgen05.cp 32x128b.warpx4: 4 columns
-//      for A, 8 for B) and issues four block-scaled MMAs (M128 x N256 x K32, scale ids 0..3) into the FP32 accumulator;
-//      the epilogue is the folded kernel's (tcgen05.ld, staging, TMA store).  The scale columns leave room for one
-//      256-column accumulator only, so a tile's epilogue does not overlap the next tile's main loop.
+//      tensor core's scale copy takes: unit (K step of 128, row tile of 128) holds byte (row r, 32-group j) at
+//      (r % 32) * 16 + (r / 32) * 4 + j; units are stored [K step][row tile], so the two units of a 256-row B tile are
+//      adjacent.
+//   2. gemm_mx_kernel: persistent, warp-specialised, one CTA pair (cta_group::2) per 256 x 256 tile.  Each CTA's TMA
+//      producer brings its 128 rows of A, its 128-row half of B, the scale unit of its A rows and both scale units of
+//      the B tile into a 5-stage ring; the leader's MMA thread copies a stage's scales to tensor memory
+//      (tcgen05.cp.cta_group::2 32x128b.warpx4: each CTA's own shared memory to its own tensor memory, 4 columns for A,
+//      8 for B) and issues four block-scaled MMAs (M256 x N256 x K32, scale ids 0..3) into the FP32 accumulator; the
+//      epilogue is the folded kernel's (tcgen05.ld, staging, TMA store).  Twelve scale columns beside a 256-column
+//      accumulator leave no room for a second accumulator in the 512 columns, so the epilogue warps first drain the
+//      whole accumulator into registers, hand it back, and only then convert and store: the next tile's main loop waits
+//      for the drain, not for the stores.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdlib.h>
@@ -26,12 +31,12 @@
 
 namespace ufp4 {
 
-constexpr int kMxStages = 3;
-constexpr int kMxA = kTM * kTK;                       // 16 KB
-constexpr int kMxB = kTN * kTK;                       // 32 KB
+constexpr int kMxStages = 5;
+constexpr int kMxA = kTM * kTK;                       // 16 KB: this CTA's 128 rows of the pair's A tile
+constexpr int kMxB = (kTN / 2) * kTK;                 // 16 KB: this CTA's 128-row half of the B tile
 constexpr int kMxSfUnit = 512;                        // scales of 128 rows x 4 groups of 32
-constexpr int kMxSfA = kMxSfUnit, kMxSfB = 2 * kMxSfUnit;
-constexpr int kMxStageBytes = kMxA + kMxB + kMxSfA + kMxSfB;      // 50688: a multiple of 1024 + 1536 -> see offsets below
+constexpr int kMxSfA = kMxSfUnit, kMxSfB = 2 * kMxSfUnit;         // own rows of A; all 256 rows of the B tile
+constexpr int kMxStageBytes = kMxA + kMxB + kMxSfA + kMxSfB;      // what one CTA's producer brings per stage
 constexpr int kMxEpiWarps = 8;
 constexpr int kMxThreads = 64 + 32 * kMxEpiWarps;
 // layout: [A tiles][B tiles][scale units][epilogue staging][barriers]; operand tiles and staging 1024-byte aligned
@@ -40,7 +45,8 @@ constexpr int kMxOffSf = kMxOffB + kMxStages * kMxB;
 constexpr int kMxOffEpi = (kMxOffSf + kMxStages * (kMxSfA + kMxSfB) + 1023) / 1024 * 1024;    // swizzled staging boxes
 constexpr int kMxOffBars = kMxOffEpi + kMxEpiWarps * 4096;
 constexpr int kMxSmem = kMxOffBars + 256;
-static_assert(kMxOffEpi % 1024 == 0 && kMxOffB % 1024 == 0 && kMxSmem <= 227 * 1024, "shared-memory layout");
+static_assert(kMxOffEpi % 1024 == 0 && kMxOffB % 1024 == 0 && kMxOffSf % 128 == 0 && kMxSmem <= 227 * 1024, "shared-memory layout");
+static_assert(16 * kMxStages + 24 <= 160, "barriers, the tensor-memory slot and the abort flag share 256 bytes");
 constexpr int kMxDMin = -14;                          // smallest exponent gap an E5M2 element still holds exactly
 
 // ------------------------------------------------------------------------------------------------------------------
@@ -53,7 +59,7 @@ struct MxOperand {
     int64_t ldc, lds, rows, rows_padded;   // rows_padded: multiple of 256 (whole scale units for every tile)
     int grid;
     uint8_t *out8;      // [rows][K]
-    uint8_t *sf;        // [rows_padded / 128][ksteps][512]
+    uint8_t *sf;        // [ksteps][rows_padded / 128][512]
 };
 
 struct MxDecodeParams {
@@ -71,7 +77,7 @@ __global__ void __launch_bounds__(256) decode_mx_kernel(const MxDecodeParams P) 
     const int64_t gid = ((int64_t)blockIdx.x - (is_b ? P.a_ctas : 0)) * 256 + threadIdx.x;
     const int64_t row = gid / ngroups, g = gid - row * ngroups;
     if (row >= O.rows_padded) return;
-    uint8_t *sf = O.sf + ((row >> 7) * P.ksteps + (g >> 2)) * kMxSfUnit + ((row & 31) << 4) + (((row >> 5) & 3) << 2) + (g & 3);
+    uint8_t *sf = O.sf + ((g >> 2) * (O.rows_padded >> 7) + (row >> 7)) * kMxSfUnit + ((row & 31) << 4) + (((row >> 5) & 3) << 2) + (g & 3);
     const int64_t nkb = P.K >> 4;
     if (row >= O.rows || 2 * g >= nkb) {
         *sf = 127;                           // padding: scale 1 on all-zero elements (the TMA fills them with zeros)
@@ -123,12 +129,6 @@ __global__ void __launch_bounds__(256) decode_mx_kernel(const MxDecodeParams P) 
 // product
 // ------------------------------------------------------------------------------------------------------------------
 
-// Untiled bulk copy global -> shared, completion on an mbarrier (both addresses 16-byte aligned, size a multiple of 16).
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
 // Shared-memory descriptor of a 512-byte scale unit for tcgen05.cp: 32 rows of 16 bytes, no swizzle, 8-row groups 128
 // bytes apart.
 __device__ __forceinline__ uint64_t sf_desc(uint32_t saddr) {
@@ -139,29 +139,32 @@ __device__ __forceinline__ uint64_t sf_desc(uint32_t saddr) {
     d |= (uint64_t)1u << 46;
     return d;
 }
+// One scale unit from shared to tensor memory, in both CTAs of the pair: each CTA copies from its own shared memory (same
+// offset) into its own tensor memory (same column); 4 columns, the 128 bytes of a 32-row group replicated to the four
+// lane quarters.
 __device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t desc) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
+    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(desc) : "memory");
 }
-// kind::mxf8f6f4, block-scaled: A = B = E5M2 (format 1), UE8M0 scales, both K-major, M = 128, N = 256; sf_id picks the byte
-// (the 32-group of the K step) of the scale columns.
+// kind::mxf8f6f4, block-scaled, on a CTA pair: A = B = E5M2 (format 1), UE8M0 scales, both K-major, M = 256, N = 256;
+// sf_id picks the byte (the 32-group of the K step) of the scale columns.
 __device__ __forceinline__ void tc_mma_mx(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t sf_id, uint32_t t_sfa,
                                           uint32_t t_sfb, uint32_t accumulate) {
     const uint32_t idesc = (sf_id << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTN >> 3) << 17) | (1u << 23) |
-                           ((uint32_t)(kTM >> 4) << 24) | (sf_id << 29);
+                           ((uint32_t)((2 * kTM) >> 4) << 24) | (sf_id << 29);
     asm volatile(
         "{ .reg .pred p; setp.ne.b32 p, %6, 0; "
-        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%4], [%5], p; }"
+        "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%4], [%5], p; }"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(t_sfa), "r"(t_sfb), "r"(accumulate) : "memory");
 }
 
 struct MxArgs {
-    const uint8_t *sfA, *sfB;    // scale units [row tile][K step][512]
-    int64_t ksteps;              // K steps per row tile in those arrays
+    int64_t a_tiles, b_tiles;    // 128-row tiles of the (padded) scale arrays: unit of (K step ks, tile t) is row ks * tiles + t
     float unit;                  // product of the two grids' code units
 };
 
 __global__ void __launch_bounds__(kMxThreads, 1)
 gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmSfA, const __grid_constant__ CUtensorMap tmSfB,
                const __grid_constant__ CUtensorMap tmC, const TcParams P, const MxArgs X) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t base = smem_u32(smem);
@@ -171,59 +174,64 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kMxOffBars + 16 * kMxStages + 16);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kMxOffBars + 160);   // flag, poll limit
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // rank 0 of the pair issues the MMAs and owns the barriers the pair synchronises on
+    const int rank = (int)cluster_cta_rank();
+    const int group_id = blockIdx.x / 2, num_groups_launched = gridDim.x / 2;
+    const uint32_t lead_full_bar = map_to_cta(full_bar, 0), lead_tempty_bar = map_to_cta(tempty_bar, 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMxStages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(full_bar + 8 * s, 2);              // one arrive.expect_tx per CTA of the pair
             mbar_init(empty_bar + 8 * s, 1);
         }
         mbar_init(tfull_bar, 1);
-        mbar_init(tempty_bar, kMxEpiWarps);
+        mbar_init(tempty_bar, 2 * kMxEpiWarps);
         abort_flag[0] = (base & 1023u) ? 1u : 0u;
         abort_flag[1] = P.wait_limit ? P.wait_limit : kWaitLimit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         __syncwarp();
-        tmem_alloc<1>(smem_u32((const void *)tmem_slot), 512);
+        tmem_alloc<2>(smem_u32((const void *)tmem_slot), 512);
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();                                  // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t t_sfa = tmem_base + kTN, t_sfb = tmem_base + kTN + 4;     // accumulator: columns 0..255, then the scales
 
     if (warp == 0) {
         if (lane == 0) {
-            // ---------------- producer: operand tiles by TMA, scale units by bulk copies
+            // ---------------- TMA producer: this CTA's rows of A and of B, the scales of its A rows and of the whole B tile
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && !P.skip_loads && tile < P.total_tiles; tile += gridDim.x) {
-                const TileInfo t = tile_info<1>(P, tile, 0);
-                const int64_t ta = t.m0 >> 7, tb = t.n0 >> 7;
+            for (int tile = group_id; ok && !P.skip_loads && tile < P.total_tiles; tile += num_groups_launched) {
+                const TileInfo t = tile_info<2>(P, tile, rank);
+                const int32_t ta = (int32_t)(t.m0 >> 7), tb = (int32_t)(t.n0 >> 7);
                 for (int kb = 0; kb < t.nkb; ++kb) {
                     if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const int64_t ks = t.kb0 + kb;
-                    const uint32_t fb = full_bar + 8 * stage, sf = sSf + stage * (kMxSfA + kMxSfB);
-                    mbar_expect_tx(fb, kMxStageBytes);
-                    tma_load_2d(sA + stage * kMxA, &tmA, (int32_t)(ks * kTK), (int32_t)t.m0, fb);
-                    tma_load_2d(sB + stage * kMxB, &tmB, (int32_t)(ks * kTK), (int32_t)t.n0, fb);
-                    bulk_load(sf, X.sfA + (ta * X.ksteps + ks) * kMxSfUnit, kMxSfUnit, fb);
-                    bulk_load(sf + kMxSfUnit, X.sfB + (tb * X.ksteps + ks) * kMxSfUnit, kMxSfUnit, fb);
-                    bulk_load(sf + 2 * kMxSfUnit, X.sfB + ((tb + 1) * X.ksteps + ks) * kMxSfUnit, kMxSfUnit, fb);
+                    const int32_t ks = t.kb0 + kb;
+                    const uint32_t fb = lead_full_bar + 8 * stage, sf = sSf + stage * (kMxSfA + kMxSfB);
+                    if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, kMxStageBytes);
+                    else mbar_expect_tx_cluster(fb, kMxStageBytes);
+                    tma_load_2d_pair(sA + stage * kMxA, &tmA, ks * kTK, (int32_t)t.m0, fb);
+                    tma_load_2d_pair(sB + stage * kMxB, &tmB, ks * kTK, (int32_t)(t.n0 + rank * (kTN / 2)), fb);
+                    tma_load_2d_pair(sf, &tmSfA, 0, (int32_t)(ks * X.a_tiles) + ta, fb);
+                    tma_load_2d_pair(sf + kMxSfUnit, &tmSfB, 0, (int32_t)(ks * X.b_tiles) + tb, fb);
                     if (++stage == kMxStages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
+        if (lane == 0 && rank == 0) {
+            // ---------------- MMA issuer (rank 0 of the pair)
             int stage = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
-                const TileInfo t = tile_info<1>(P, tile, 0);
+            for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+                const TileInfo t = tile_info<2>(P, tile, rank);
                 if (t.nkb == 0) continue;
                 if (!mbar_wait(tempty_bar, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -239,58 +247,57 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int k = 0; k < 4; ++k)
                         tc_mma_mx(tmem_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), (uint32_t)k, t_sfa, t_sfb,
                                   (kb > 0 || k > 0) ? 1u : 0u);
-                    tc_commit<1>(empty_bar + 8 * stage);
+                    tc_commit<2>(empty_bar + 8 * stage);   // the stage is free in both CTAs once read
                     if (++stage == kMxStages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit<1>(tfull_bar);
+                tc_commit<2>(tfull_bar);                   // accumulator complete, in both CTAs
                 acc_phase ^= 1u;
             }
         }
     } else {
-        // ---------------- epilogue: TMEM -> registers -> x unit -> staging -> TMA store
+        // ---------------- epilogue: TMEM -> registers (all of this warp's four boxes) -> accumulator handed back ->
+        // x unit -> staging -> TMA store
         const int q = warp & 3, half = (warp - 2) >> 2;
         uint8_t *buf = smem + kMxOffEpi + (warp - 2) * 4096;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
-            const TileInfo t = tile_info<1>(P, tile, 0);
+        for (int tile = group_id; ok && tile < P.total_tiles; tile += num_groups_launched) {
+            const TileInfo t = tile_info<2>(P, tile, rank);
             const int64_t m_own = t.m0 + q * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(4 * half * 32);
+            uint32_t v[4][32];
             if (t.nkb > 0) {
                 if (!mbar_wait_warp(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 acc_phase ^= 1u;
-            }
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            const int32_t c_row = (int32_t)(t.m0 + q * 32), c_grp = (int32_t)(t.c_row0 / (P.M > 0 ? P.M : 1));
-#pragma unroll 1
-            for (int cc = 0; cc < 4; ++cc) {
-                const int c = 4 * half + cc;
-                uint32_t v[32];
-                if (t.nkb > 0) {
-                    tc_ld32(taddr + (uint32_t)(c * 32), v);
-                    tc_wait_ld();
-                    if (cc == 3) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(tempty_bar);
-                    }
-                } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = 0u;
-                }
-                const int64_t n_base = t.n0 + c * 32;
+                for (int cc = 0; cc < 4; ++cc) tc_ld32(taddr + (uint32_t)(cc * 32), v[cc]);
+                tc_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(lead_tempty_bar);
+            } else {
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[cc][j] = 0u;
+            }
+            const int32_t c_row = (int32_t)(t.m0 + q * 32), c_grp = (int32_t)(t.c_row0 / (P.M > 0 ? P.M : 1));
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                const int64_t n_base = t.n0 + (4 * half + cc) * 32;
                 if (n_base >= P.N || c_row >= t.row_end) continue;
                 float x[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(v[j]) * X.unit;
+                for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(v[cc][j]) * X.unit;
                 if (n_base + 32 > P.N && P.n_unaligned) epi_store_box_plain(P, x, t.c_row0 + m_own, n_base, m_own < t.row_end);
                 else epi_store_box_tma(P, &tmC, buf, lane, x, (int32_t)n_base, c_row, c_grp);
             }
         }
         epi_store_drain(lane);
     }
-    tc_teardown<1>(abort_flag, P.dev_status, tmem_base, 512, warp);
+    tc_teardown<2>(abort_flag, P.dev_status, tmem_base, 512, warp);
 }
 
 // ------------------------------------------------------------------------------------------------------------------
@@ -330,6 +337,19 @@ static bool mx_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Scale units as a matrix of 32-bit words: one unit (512 bytes) per row, `units_per_box` consecutive units per copy.
+static bool mx_make_sf_map(CUtensorMap *map, const void *ptr, int64_t units, int units_per_box) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)(kMxSfUnit / 4), (cuuint64_t)units};
+    cuuint64_t strides[1] = {(cuuint64_t)kMxSfUnit};
+    cuuint32_t box[2] = {(cuuint32_t)(kMxSfUnit / 4), (cuuint32_t)units_per_box};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode, int64_t M,
                    int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n, void *workspace,
                    size_t workspace_bytes, int32_t *dev_status, void *stream) {
@@ -356,8 +376,12 @@ int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_
     decode_mx_kernel<<<(unsigned)ctas, 256, 0, st>>>(D);
     if (cudaGetLastError() != cudaSuccess) return UFP4_ERR_CUDA;
 
-    CUtensorMap tmA, tmB, tmC = {};
-    if (!mx_make_map(&tmA, A8, A->rows, K, kTM) || !mx_make_map(&tmB, B8, B->rows, K, kTN)) return UFP4_ERR_CUDA;
+    const int64_t a_tiles = mx_pad_rows(A->rows) / 128, b_tiles = mx_pad_rows(B->rows) / 128;
+    if (ksteps * a_tiles > 0x7FFFFFFF || ksteps * b_tiles > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
+    CUtensorMap tmA, tmB, tmSfA, tmSfB, tmC = {};
+    if (!mx_make_map(&tmA, A8, A->rows, K, kTM) || !mx_make_map(&tmB, B8, B->rows, K, kTN / 2) ||
+        !mx_make_sf_map(&tmSfA, sfA, ksteps * a_tiles, 1) || !mx_make_sf_map(&tmSfB, sfB, ksteps * b_tiles, 2))
+        return UFP4_ERR_CUDA;
     {
         EncodeTiledFn fn = encode_tiled_fn();
         if (!fn) return UFP4_ERR_CUDA;
@@ -378,7 +402,7 @@ int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_
     P.M = M; P.N = N; P.K = K; P.mode = mode;
     P.offsets = offsets; P.num_groups = num_groups; P.group_n = group_n;
     P.dev_status = dev_status;
-    P.mt = (int)((M + kTM - 1) / kTM);
+    P.mt = (int)((M + 2 * kTM - 1) / (2 * kTM));
     P.nt = (int)((N + kTN - 1) / kTN);
     const int64_t total = (int64_t)P.mt * P.nt * (mode == 2 ? num_groups : 1);
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
@@ -387,7 +411,7 @@ int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_
     P.wait_limit = debug_wait_limit();
     P.skip_loads = debug_skip_loads();
     MxArgs X = {};
-    X.sfA = sfA; X.sfB = sfB; X.ksteps = ksteps;
+    X.a_tiles = a_tiles; X.b_tiles = b_tiles;
     auto unit_of = [](int grid) { return codebook_of(grid) == UFP4_GRID_INT4 ? 1.0f : (codebook_of(grid) == UFP4_GRID_E1M2 ? 0.25f : 0.5f); };
     X.unit = unit_of(A->grid) * unit_of(B->grid);
 
@@ -396,12 +420,21 @@ int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_
     const int rc_setup = device_setup(slots, [](int ordinal, DeviceSetup &d) -> int {
         UFP4_CUDA_OK(cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, ordinal));
         UFP4_CUDA_OK(cudaFuncSetAttribute(gemm_mx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMxSmem));
+        d.max_pairs = resident_pairs(gemm_mx_kernel, kMxThreads, kMxSmem, d.num_sms);
         return UFP4_OK;
     }, &dev);
     if (rc_setup != UFP4_OK) return rc_setup;
-    const int grid = (int)(total < dev->num_sms ? total : dev->num_sms);
-    gemm_mx_kernel<<<grid, kMxThreads, kMxSmem, st>>>(tmA, tmB, tmC, P, X);
-    return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(2 * (unsigned)(total < dev->max_pairs ? total : dev->max_pairs));
+    cfg.blockDim = dim3(kMxThreads);
+    cfg.dynamicSmemBytes = kMxSmem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_mx_kernel, tmA, tmB, tmSfA, tmSfB, tmC, P, X) == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 
 }  // namespace ufp4

@@ -15,14 +15,15 @@ from test_gpu_gemm import grouped_reference
 pytestmark = pytest.mark.gpu
 
 
-def test_auto_takes_mx_for_two_1x32_tensors():
+def test_mx_is_taken_on_request_and_auto_keeps_the_folded_path():
     X, W = inputs.normal_bf16(64, 64, 1.0, seed=1), inputs.normal_bf16(32, 64, 0.02, seed=2)
     kw = dict(rht_block=16, seed_rht=3)
     A32 = to_device(oracle_quantize(X, oracle.AXIS_ROW, scale_fmt=oracle.SCALE_E8M0_B32, **kw))
     B32 = to_device(oracle_quantize(W, oracle.AXIS_ROW, scale_fmt=oracle.SCALE_E8M0_B32, **kw))
     B16 = to_device(oracle_quantize(W, oracle.AXIS_ROW, scale_fmt=oracle.SCALE_POW2, **kw))
     BF = to_device(oracle_quantize(W, oracle.AXIS_ROW, scale_fmt=oracle.SCALE_FP32, **kw))
-    assert ufp4.gemm_path_taken(A32, B32, ufp4.PATH_AUTO) == (ufp4.PATH_MX, 2) and ufp4.gemm_path_name(A32, B32) == "mx"
+    assert ufp4.gemm_path_taken(A32, B32, ufp4.PATH_MX) == (ufp4.PATH_MX, 2) and ufp4.gemm_path_name(A32, B32, ufp4.PATH_MX) == "mx"
+    assert ufp4.gemm_path_taken(A32, B32, ufp4.PATH_AUTO)[0] == ufp4.PATH_TENSOR
     assert ufp4.gemm_path_taken(A32, B16, ufp4.PATH_AUTO)[0] == ufp4.PATH_TENSOR
     assert ufp4.gemm_path_taken(A32, B16, ufp4.PATH_MX)[0] == ufp4.PATH_MX
     with pytest.raises(ufp4.Ufp4Error) as e:
@@ -33,7 +34,8 @@ def test_auto_takes_mx_for_two_1x32_tensors():
 @pytest.mark.parametrize("fmt", [oracle.SCALE_E8M0_B32, oracle.SCALE_POW2])
 @pytest.mark.parametrize("grids", [(oracle.GRID_INT4, oracle.GRID_INT4), (oracle.GRID_E1M2, oracle.GRID_E2M1)])
 @pytest.mark.parametrize("shape", [(256, 256, 256), (128, 256, 128), (200, 72, 160), (1, 1, 32), (130, 260, 192),
-                                   (384, 520, 1056), (1024, 1536, 2048), (640, 300, 8192)])
+                                   (384, 520, 1056), (1024, 1536, 2048), (640, 300, 8192),
+                                   (2304, 2560, 160)])                     # more tiles than resident CTA pairs
 def test_shapes_grids_and_scale_formats(shape, grids, fmt):
     M, N, K = shape
     X = inputs.heavy_tailed_activations(M, K, seed=21 + M)
@@ -76,7 +78,7 @@ def test_a_row_whose_scales_spread_over_2_to_the_30_is_exact_here_and_flagged_on
     A, B = oracle_quantize(X, oracle.AXIS_ROW, **kw), oracle_quantize(W, oracle.AXIS_ROW, **kw)
     ref, S = oracle.gemm(A, B)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    got = ufp4.gemm(to_device(A), to_device(B), dev_status=status)                 # AUTO: MX
+    got = ufp4.gemm(to_device(A), to_device(B), path=ufp4.PATH_MX, dev_status=status)
     assert int(status.item()) == 0
     assert_gemm_close(got.cpu().numpy(), ref, S, "2^30 spread, hardware scales")
     # each small group on its own: exact as well (the large group does not mask them)
