@@ -173,8 +173,8 @@ int ufp4_selftest_division(int32_t *dev_mismatches, void *stream);
 size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, int path);
 
 /* GEMM paths (given a workspace of ufp4_gemm_workspace_bytes(A, B, path); without one AUTO falls back to EXACT).
- * AUTO:    TENSOR when both operands use power-of-two scales (1 x 16 or 1 x 32), FP16 when both use E4M3 x tensor
- *          scales, else SPLIT.
+ * AUTO:    TENSOR when both operands use power-of-two scales (1 x 16 or 1 x 32); when both use E4M3 x tensor scales, NVF4
+ *          for a plain product with an E2M1 tensor in it and FP16 otherwise; else SPLIT.
  * EXACT:   CUDA-core kernel: integer block partials (dp4a) promoted with the two FP32 block scales, FP64 running sum;
  *          every grid and scale format, no workspace; the slow reference path.
  * TENSOR:  tcgen05 / TMEM kernel on 8-bit floating-point operands into which code x 2^e is folded exactly (POW2 scales
@@ -200,10 +200,16 @@ size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, i
  *          more than 2^14 below its neighbour is flushed and sets UFP4_DEV_EXP_WINDOW).  Plain and reduction-grouped
  *          products; a row-grouped product returns UFP4_ERR_UNSUPPORTED.  On request only: on the same operands TENSOR
  *          is the faster path (its accumulators are double-buffered and it copies no scales inside the main loop), so
- *          MX is the choice for rows whose block exponents spread beyond TENSOR's window. */
+ *          MX is the choice for rows whose block exponents spread beyond TENSOR's window.
+ * NVF4:    tcgen05 / TMEM kernel on the FP4 tensor path (kind::mxf4nvf4) with the hardware applying one UE4M3 scale per
+ *          16 elements, for operands that BOTH carry E4M3 block scales times a per-tensor FP32 scale.  That path knows
+ *          the E2M1 levels only (Sec. 1): an E2M1 tensor is read as it stands (one MMA per 64-element step, nothing is
+ *          decoded but the scale layout), a uniform code q is split into two E2M1 values, q / 2 = hi + lo, and the
+ *          product taken plane by plane (four MMAs per step for two uniform tensors, two when one of them is E2M1).
+ *          Exact like FP16 (no window, the tensor scales multiply the result once).  Plain products only. */
 typedef enum {
     UFP4_PATH_AUTO = 0, UFP4_PATH_EXACT = 1, UFP4_PATH_TENSOR = 2, UFP4_PATH_PROMOTE = 3, UFP4_PATH_SPLIT = 4,
-    UFP4_PATH_FP16 = 5, UFP4_PATH_MX = 6
+    UFP4_PATH_FP16 = 5, UFP4_PATH_MX = 6, UFP4_PATH_NVF4 = 7
 } ufp4_gemm_path;
 
 /* Which path ufp4_gemm would take for these operands and this request (given a sufficient workspace), or a negative

@@ -18,7 +18,7 @@ AXIS_ROW, AXIS_COL, AXIS_BOTH = 0, 1, 2
 SCALE_FP32, SCALE_POW2, SCALE_E4M3_TENSOR = 0, 1, 2
 SCALE_E8M0_B32 = 3      # one power-of-two scale per 32 elements (MXFP4's block layout), read by the GEMMs like POW2
 FWD_Y, BWD_DX, BWD_DW = 0, 1, 2
-PATH_AUTO, PATH_EXACT, PATH_TENSOR, PATH_PROMOTE, PATH_SPLIT, PATH_FP16, PATH_MX = 0, 1, 2, 3, 4, 5, 6
+PATH_AUTO, PATH_EXACT, PATH_TENSOR, PATH_PROMOTE, PATH_SPLIT, PATH_FP16, PATH_MX, PATH_NVF4 = 0, 1, 2, 3, 4, 5, 6, 7
 DEV_NONFINITE, DEV_EXP_WINDOW, DEV_WAIT_TIMEOUT = 1, 2, 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -292,7 +292,7 @@ def gemm_launch_count(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> int:
 
 
 def gemm_path_name(A: QTensor, B: QTensor, path: int = PATH_AUTO) -> str:
-    return {PATH_EXACT: "exact", PATH_TENSOR: "tensor", PATH_PROMOTE: "promote", PATH_SPLIT: "split", PATH_FP16: "fp16", PATH_MX: "mx"}[gemm_path_taken(A, B, path)[0]]
+    return {PATH_EXACT: "exact", PATH_TENSOR: "tensor", PATH_PROMOTE: "promote", PATH_SPLIT: "split", PATH_FP16: "fp16", PATH_MX: "mx", PATH_NVF4: "nvf4"}[gemm_path_taken(A, B, path)[0]]
 
 
 def _alloc_out(rows: int, cols: int, bf16: bool, device) -> torch.Tensor:

@@ -52,6 +52,11 @@ bool gemm_mx_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, 
 int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int mode, int64_t M,
                    int64_t N, int64_t K, const int64_t *offsets, int num_groups, int64_t group_n, void *workspace,
                    size_t workspace_bytes, int32_t *dev_status, void *stream);
+size_t gemm_nvf4_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B);
+int gemm_nvf4_kernel_launches();
+bool gemm_nvf4_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
+int gemm_nvf4_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_t ldc, int c_is_bf16, int64_t M, int64_t N,
+                     int64_t K, void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
 size_t gemm_fp16_workspace_bytes(int64_t a_rows, int64_t b_rows, int64_t K);
 bool gemm_fp16_supported(const ufp4_qtensor *A, const ufp4_qtensor *B, int64_t M, int64_t N, int64_t K, int mode);
 
@@ -70,7 +75,7 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                          int mode, int64_t M, int64_t N, int64_t K, const int64_t *offsets, const int64_t *host_offsets,
                          int num_groups, int64_t group_n, void *workspace, size_t workspace_bytes, int32_t *dev_status,
                          void *stream) {
-    if (path < 0 || path > 6) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 7) return UFP4_ERR_ENUM;
     if (!C) return UFP4_ERR_NULL;
     if (ldc < N) return UFP4_ERR_SHAPE;
     if (!aligned_to(C, 16) || (ldc * (c_is_bf16 ? 2 : 4)) % 16 != 0) return UFP4_ERR_ALIGN;
@@ -91,6 +96,16 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
             return gemm_tensor_launch(A, B, C, ldc, c_is_bf16, mode, M, N, K, offsets, host_offsets, num_groups, group_n,
                                       workspace, workspace_bytes, dev_status, stream, nullptr);
         if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
+    }
+    // NVF4 (native FP4 with hardware UE4M3 scales): E4M3 x tensor scales on both operands, plain products.  On request, and
+    // what AUTO takes when an operand is an E2M1 tensor (one or two MMAs per step at the FP4 rate: faster than FP16)
+    const bool nvf4_ok = gemm_nvf4_supported(A, B, M, N, K, mode);
+    const bool nvf4_auto = nvf4_ok && (codebook_of(A->grid) == UFP4_GRID_E2M1 || codebook_of(B->grid) == UFP4_GRID_E2M1);
+    if (path == UFP4_PATH_NVF4 && !nvf4_ok) return UFP4_ERR_UNSUPPORTED;
+    if (path == UFP4_PATH_NVF4 || (path == UFP4_PATH_AUTO && nvf4_auto)) {
+        if (workspace && workspace_bytes >= gemm_nvf4_workspace_bytes(A, B))
+            return gemm_nvf4_launch(A, B, C, ldc, c_is_bf16, M, N, K, workspace, workspace_bytes, dev_status, stream);
+        if (path == UFP4_PATH_NVF4) return UFP4_ERR_WORKSPACE;
     }
     // FP16 (one piece): E4M3 x tensor scales on both operands
     const bool fp16_ok = gemm_fp16_supported(A, B, M, N, K, mode);
@@ -160,6 +175,7 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     if (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && pow2))
         return pow2 ? ufp4::gemm_tensor_workspace_bytes(A->rows, B->rows, A->k) : 0;
     const bool e4m3 = A->scale_fmt == UFP4_SCALE_E4M3_TENSOR && B->scale_fmt == UFP4_SCALE_E4M3_TENSOR;
+    if (path == UFP4_PATH_NVF4) return e4m3 ? ufp4::gemm_nvf4_workspace_bytes(A, B) : 0;
     if (path == UFP4_PATH_FP16) return e4m3 ? ufp4::gemm_fp16_workspace_bytes(A->rows, B->rows, A->k) : 0;
     // AUTO takes FP16 for E4M3 x tensor scales, else SPLIT, and PROMOTE only where SPLIT does not apply: the two-piece
     // workspace is enough for all of them
@@ -167,7 +183,9 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     const size_t promote = ufp4::gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
     if (path == UFP4_PATH_SPLIT) return split;
     if (path == UFP4_PATH_PROMOTE) return promote;
-    return split > promote ? split : promote;
+    const size_t nvf4 = e4m3 ? ufp4::gemm_nvf4_workspace_bytes(A, B) : 0;      // what AUTO takes when an operand is an E2M1 tensor
+    const size_t m = split > promote ? split : promote;
+    return m > nvf4 ? m : nvf4;
 }
 
 extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B, int path, int *kernel_launches) {
@@ -175,22 +193,27 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     if (rc != UFP4_OK) return rc;
     rc = ufp4::check_operand(B);
     if (rc != UFP4_OK) return rc;
-    if (path < 0 || path > 6) return UFP4_ERR_ENUM;
+    if (path < 0 || path > 7) return UFP4_ERR_ENUM;
     if (A->k != B->k) return UFP4_ERR_SHAPE;
     if (path == UFP4_PATH_MX && !ufp4::gemm_mx_supported(A, B, A->rows, B->rows, A->k, 0)) return UFP4_ERR_UNSUPPORTED;
     bool tensor_ok = ufp4::gemm_tensor_supported(A, B, A->rows, B->rows, A->k, 0);
     bool split_ok = ufp4::gemm_split_supported(A, B, A->rows, B->rows, A->k, 0);
     bool fp16_ok = ufp4::gemm_fp16_supported(A, B, A->rows, B->rows, A->k, 0);
+    bool nvf4_ok = ufp4::gemm_nvf4_supported(A, B, A->rows, B->rows, A->k, 0);
+    bool nvf4_auto = nvf4_ok && (ufp4::codebook_of(A->grid) == UFP4_GRID_E2M1 || ufp4::codebook_of(B->grid) == UFP4_GRID_E2M1);
+    if (path == UFP4_PATH_NVF4 && !nvf4_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_FP16 && !fp16_ok) return UFP4_ERR_UNSUPPORTED;
     int taken = path == UFP4_PATH_EXACT ? UFP4_PATH_EXACT
               : path == UFP4_PATH_MX ? UFP4_PATH_MX
               : (path == UFP4_PATH_TENSOR || (path == UFP4_PATH_AUTO && tensor_ok)) ? UFP4_PATH_TENSOR
+              : (path == UFP4_PATH_NVF4 || (path == UFP4_PATH_AUTO && nvf4_auto)) ? UFP4_PATH_NVF4
               : (path == UFP4_PATH_FP16 || (path == UFP4_PATH_AUTO && fp16_ok)) ? UFP4_PATH_FP16
               : (path == UFP4_PATH_SPLIT || (path == UFP4_PATH_AUTO && split_ok)) ? UFP4_PATH_SPLIT : UFP4_PATH_PROMOTE;
     if (kernel_launches)
         *kernel_launches = taken == UFP4_PATH_EXACT ? 1 : taken == UFP4_PATH_MX ? ufp4::gemm_mx_kernel_launches()
+                         : taken == UFP4_PATH_NVF4 ? ufp4::gemm_nvf4_kernel_launches()
                          : taken == UFP4_PATH_TENSOR ? ufp4::gemm_tensor_kernel_launches()
                          : (taken == UFP4_PATH_SPLIT || taken == UFP4_PATH_FP16) ? ufp4::gemm_split_kernel_launches()
                                                     : ufp4::gemm_promote_kernel_launches();
