@@ -174,7 +174,7 @@ size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qtensor *B, i
 
 /* GEMM paths (given a workspace of ufp4_gemm_workspace_bytes(A, B, path); without one AUTO falls back to EXACT).
  * AUTO:    TENSOR when both operands use power-of-two scales (1 x 16 or 1 x 32); when both use E4M3 x tensor scales, NVF4
- *          for a plain product with an E2M1 tensor in it and FP16 otherwise; else SPLIT.
+ *          for plain products and FP16 for grouped ones; else SPLIT.
  * EXACT:   CUDA-core kernel: integer block partials (dp4a) promoted with the two FP32 block scales, FP64 running sum;
  *          every grid and scale format, no workspace; the slow reference path.
  * TENSOR:  tcgen05 / TMEM kernel on 8-bit floating-point operands into which code x 2^e is folded exactly (POW2 scales

@@ -97,10 +97,10 @@ static int gemm_dispatch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, 
                                       workspace, workspace_bytes, dev_status, stream, nullptr);
         if (path == UFP4_PATH_TENSOR) return UFP4_ERR_WORKSPACE;
     }
-    // NVF4 (native FP4 with hardware UE4M3 scales): E4M3 x tensor scales on both operands, plain products.  On request, and
-    // what AUTO takes when an operand is an E2M1 tensor (one or two MMAs per step at the FP4 rate: faster than FP16)
+    // NVF4 (native FP4 with hardware UE4M3 scales): E4M3 x tensor scales on both operands, plain products; what AUTO takes
+    // for those (measured faster than FP16 with one, two or four MMAs per step)
     const bool nvf4_ok = gemm_nvf4_supported(A, B, M, N, K, mode);
-    const bool nvf4_auto = nvf4_ok && (codebook_of(A->grid) == UFP4_GRID_E2M1 || codebook_of(B->grid) == UFP4_GRID_E2M1);
+    const bool nvf4_auto = nvf4_ok;
     if (path == UFP4_PATH_NVF4 && !nvf4_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_NVF4 || (path == UFP4_PATH_AUTO && nvf4_auto)) {
         if (workspace && workspace_bytes >= gemm_nvf4_workspace_bytes(A, B))
@@ -183,7 +183,7 @@ extern "C" size_t ufp4_gemm_workspace_bytes(const ufp4_qtensor *A, const ufp4_qt
     const size_t promote = ufp4::gemm_promote_workspace_bytes(A->rows, B->rows, A->k);
     if (path == UFP4_PATH_SPLIT) return split;
     if (path == UFP4_PATH_PROMOTE) return promote;
-    const size_t nvf4 = e4m3 ? ufp4::gemm_nvf4_workspace_bytes(A, B) : 0;      // what AUTO takes when an operand is an E2M1 tensor
+    const size_t nvf4 = e4m3 ? ufp4::gemm_nvf4_workspace_bytes(A, B) : 0;      // what AUTO takes for plain products
     const size_t m = split > promote ? split : promote;
     return m > nvf4 ? m : nvf4;
 }
@@ -200,7 +200,7 @@ extern "C" int ufp4_gemm_path_taken(const ufp4_qtensor *A, const ufp4_qtensor *B
     bool split_ok = ufp4::gemm_split_supported(A, B, A->rows, B->rows, A->k, 0);
     bool fp16_ok = ufp4::gemm_fp16_supported(A, B, A->rows, B->rows, A->k, 0);
     bool nvf4_ok = ufp4::gemm_nvf4_supported(A, B, A->rows, B->rows, A->k, 0);
-    bool nvf4_auto = nvf4_ok && (ufp4::codebook_of(A->grid) == UFP4_GRID_E2M1 || ufp4::codebook_of(B->grid) == UFP4_GRID_E2M1);
+    bool nvf4_auto = nvf4_ok;
     if (path == UFP4_PATH_NVF4 && !nvf4_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_TENSOR && !tensor_ok) return UFP4_ERR_UNSUPPORTED;
     if (path == UFP4_PATH_SPLIT && !split_ok) return UFP4_ERR_UNSUPPORTED;

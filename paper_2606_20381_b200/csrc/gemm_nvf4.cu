@@ -117,17 +117,30 @@ __global__ void __launch_bounds__(256) decode_nvf4_kernel(const NvDecodeParams P
     *sf = sw;
     if (O.hi == nullptr) return;             // E2M1 tensors: the product kernel reads their codes in place
     const bool int4 = O.grid == UFP4_GRID_INT4;
-    const uint2 *cp = reinterpret_cast<const uint2 *>(O.codes + row * O.ldc) + 4 * c;
-    uint2 *hp = reinterpret_cast<uint2 *>(O.hi + row * P.pitch) + 4 * c, *lp = reinterpret_cast<uint2 *>(O.lo + row * P.pitch) + 4 * c;
+    const uint8_t *cp = O.codes + row * O.ldc + 32 * c;
+    uint8_t *hp = O.hi + row * P.pitch + 32 * c, *lp = O.lo + row * P.pitch + 32 * c;
+    if (4 * c + 4 <= nkb) {
+        // a whole step: two 16-byte loads, two 16-byte stores per plane (rows and steps are 16-byte aligned)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        if (4 * c + j >= nkb) break;
-        const uint2 w = __ldg(cp + j);
+        for (int j = 0; j < 2; ++j) {
+            const uint4 w = __ldg(reinterpret_cast<const uint4 *>(cp) + j);
+            uint4 h, l;
+            split_uniform8(w.x, int4, &h.x, &l.x);
+            split_uniform8(w.y, int4, &h.y, &l.y);
+            split_uniform8(w.z, int4, &h.z, &l.z);
+            split_uniform8(w.w, int4, &h.w, &l.w);
+            reinterpret_cast<uint4 *>(hp)[j] = h;
+            reinterpret_cast<uint4 *>(lp)[j] = l;
+        }
+        return;
+    }
+    for (int j = 0; 4 * c + j < nkb; ++j) {          // the last step of a row whose K is not a multiple of 64
+        const uint2 w = __ldg(reinterpret_cast<const uint2 *>(cp) + j);
         uint2 h, l;
         split_uniform8(w.x, int4, &h.x, &l.x);
         split_uniform8(w.y, int4, &h.y, &l.y);
-        hp[j] = h;
-        lp[j] = l;
+        reinterpret_cast<uint2 *>(hp)[j] = h;
+        reinterpret_cast<uint2 *>(lp)[j] = l;
     }
 }
 

@@ -24,11 +24,11 @@ def _quantize(x, axis, grid, gmax, **extra):
                            tensor_scale=_ts(x, gmax), **extra)
 
 
-def test_auto_takes_the_fp16_path_for_e4m3_tensor_scales_only():
+def test_the_fp16_path_takes_e4m3_tensor_scales_only():
     X, W = inputs.normal_bf16(64, 64, 1.0, seed=1), inputs.normal_bf16(32, 64, 0.02, seed=2)
     A, B = to_device(_quantize(X, oracle.AXIS_ROW, oracle.GRID_INT4, 7)), to_device(_quantize(W, oracle.AXIS_ROW, oracle.GRID_INT4, 7))
-    assert ufp4.gemm_path_taken(A, B, ufp4.PATH_AUTO) == (ufp4.PATH_FP16, 2)
-    assert ufp4.gemm_path_name(A, B) == "fp16"
+    assert ufp4.gemm_path_taken(A, B, ufp4.PATH_FP16) == (ufp4.PATH_FP16, 2)
+    assert ufp4.gemm_path_name(A, B, ufp4.PATH_FP16) == "fp16"
     assert ufp4.gemm_workspace_bytes(A, B, ufp4.PATH_FP16) < ufp4.gemm_workspace_bytes(A, B, ufp4.PATH_SPLIT)
     P = to_device(oracle_quantize(W, oracle.AXIS_ROW, rht_block=16, scale_fmt=oracle.SCALE_POW2, seed_rht=3))
     with pytest.raises(ufp4.Ufp4Error) as e:

@@ -31,9 +31,8 @@ def test_path_selection():
     Au, Bu = to_device(_quantize(X, oracle.AXIS_ROW, oracle.GRID_INT4)), to_device(_quantize(W, oracle.AXIS_ROW, oracle.GRID_INT4))
     Ae, Be = to_device(_quantize(X, oracle.AXIS_ROW, oracle.GRID_E2M1)), to_device(_quantize(W, oracle.AXIS_ROW, oracle.GRID_E2M1))
     assert ufp4.gemm_path_taken(Au, Bu, ufp4.PATH_NVF4) == (ufp4.PATH_NVF4, 2) and ufp4.gemm_path_name(Au, Bu, ufp4.PATH_NVF4) == "nvf4"
-    assert ufp4.gemm_path_taken(Au, Bu, ufp4.PATH_AUTO)[0] == ufp4.PATH_FP16           # uniform codes: FP16 stays the default
-    assert ufp4.gemm_path_taken(Ae, Be, ufp4.PATH_AUTO)[0] == ufp4.PATH_NVF4           # two E2M1 tensors: the FP4 path as it is
-    assert ufp4.gemm_path_taken(Au, Be, ufp4.PATH_AUTO)[0] == ufp4.PATH_NVF4           # one E2M1 tensor: two MMAs per step
+    for a, b in ((Au, Bu), (Ae, Be), (Au, Be)):          # four, one, two MMAs per step: AUTO's path for plain products
+        assert ufp4.gemm_path_taken(a, b, ufp4.PATH_AUTO)[0] == ufp4.PATH_NVF4
     # E2M1 tensors need no planes: only the scale units
     assert ufp4.gemm_workspace_bytes(Ae, Be, ufp4.PATH_NVF4) < ufp4.gemm_workspace_bytes(Au, Bu, ufp4.PATH_NVF4)
     P = to_device(oracle_quantize(W, oracle.AXIS_ROW, rht_block=16, scale_fmt=oracle.SCALE_POW2, seed_rht=3))
