@@ -94,15 +94,21 @@ class Ufp4Linear(_Ufp4Step):
 
     def __init__(self, tokens: int, in_features: int, out_features: int, device="cuda", grid: int = ufp4.GRID_INT4,
                  scale_fmt: int = ufp4.SCALE_FP32, path: int = ufp4.PATH_AUTO, rht_block: int = 16,
-                 seed_rht: int = 1, seed_sr: int = 2, out_bf16: bool = False, overlap: bool = False):
+                 seed_rht: int = 1, seed_sr: int = 2, out_bf16: bool = False, overlap: bool = False,
+                 tensor_scales=None):
+        """tensor_scales: (ts_X, ts_W, ts_dY), the per-tensor FP32 scales of the two-level E4M3 format (floats or
+        one-element device tensors); each must bound its tensor's rotated values, ts >= 4 amax / (g_max 448)."""
         T, K, N = tokens, in_features, out_features
         self.T, self.K, self.N = T, K, N
         self.grid, self.scale_fmt, self.path, self.rht_block = grid, scale_fmt, path, rht_block
         self.seed_rht, self.seed_sr = seed_rht, seed_sr
-        a = lambda r, k: ufp4.alloc_qtensor(r, k, grid, scale_fmt, device)
-        self.Xr, self.Xc = a(T, K), a(K, T)
-        self.Wr, self.Wc = a(N, K), a(K, N)
-        self.Gr, self.Gc = a(T, N), a(N, T)
+        if scale_fmt == ufp4.SCALE_E4M3_TENSOR and tensor_scales is None:
+            raise ValueError("E4M3_TENSOR needs tensor_scales = (ts_X, ts_W, ts_dY)")
+        tsx, tsw, tsg = tensor_scales if scale_fmt == ufp4.SCALE_E4M3_TENSOR else (None, None, None)
+        a = lambda r, k, ts: ufp4.alloc_qtensor(r, k, grid, scale_fmt, device, ts)
+        self.Xr, self.Xc = a(T, K, tsx), a(K, T, tsx)
+        self.Wr, self.Wc = a(N, K, tsw), a(K, N, tsw)
+        self.Gr, self.Gc = a(T, N, tsg), a(N, T, tsg)
         dt = torch.bfloat16 if out_bf16 else torch.float32
         self.Y = torch.empty(T, N, dtype=dt, device=device)
         self.dX = torch.empty(T, K, dtype=dt, device=device)

@@ -21,7 +21,8 @@ def test_tiny_workload_prints_one_complete_json_line():
     d = json.loads(lines[0])
     for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
                 "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks",
-                "sustained", "quantize_sweep", "tensor_peak_8bit_measured", "roofline_quantize", "fp32_block_scales"):
+                "sustained", "quantize_sweep", "tensor_peak_8bit_measured", "roofline_quantize", "fp32_block_scales",
+                "e4m3_tensor_scales"):
         assert key in d, key
     assert d["n_gpus"] == 1 and d["steps"] == 3 and d["value"] > 0 and d["vs_baseline"] is None and d["dev_status"] == 0
     assert d["config"]["workload"] == "tiny" and d["data"] == "synthetic"
@@ -39,6 +40,10 @@ def test_tiny_workload_prints_one_complete_json_line():
     # Table 1's FP32 block scales beside the headline, with a roofline of their own
     f32 = d["fp32_block_scales"]
     assert f32["scale_fmt"] == "fp32" and f32["roofline"]["frac"] > 0 and f32["dev_status"] == 0
+    # the two-level scale format on the FP4 pipe: the uniform grid and the E2M1 baseline grid
+    e8 = d["e4m3_tensor_scales"]
+    for g in ("uniform_int4", "e2m1_baseline"):
+        assert e8[g]["gemm_path"] == "nvf4" and e8[g]["value"] > 0 and e8[g]["dev_status"] == 0 and "clocks" in e8[g]
     # BASELINE config 3 in brief: four sizes, uniform grid and E2M1, RTNE and SR, RHT off and on
     sw = d["quantize_sweep"]
     assert [(e["rows"], e["cols"]) for e in sw] == [(4096, 4096), (8192, 8192), (16384, 8192), (32768, 8192)]

@@ -122,3 +122,29 @@ def test_grouped_products_are_refused():
     with pytest.raises(ufp4.Ufp4Error) as e:
         ufp4.gemm_grouped(A, B, off.cuda(), off, 48, ufp4.FWD_Y, path=ufp4.PATH_NVF4)
     assert e.value.status == -5
+
+
+@pytest.mark.parametrize("grid", [oracle.GRID_INT4, oracle.GRID_E1M2, oracle.GRID_E2M1])
+def test_tiny_layer_step_with_two_level_scales(grid):
+    """The tiny single-layer check in its two-level scale format (E4M3 per block, FP32 per tensor), through the recipe class:
+    the six quantized tensors bit-equal to the oracle's, the three products (AUTO: the FP4 path) within the bound."""
+    from helpers import assert_qtensor_equal
+    from paper_2606_20381_b200.recipe import Ufp4Linear
+    X, W, dY = inputs.tiny_layer(0)
+    ts = tuple(_ts(t, GMAX[grid]) for t in (X, W, dY))
+    step = Ufp4Linear(X.shape[0], X.shape[1], W.shape[0], grid=grid, scale_fmt=ufp4.SCALE_E4M3_TENSOR, tensor_scales=ts)
+    Y, dX, dW = step.step(X.cuda(), W.cuda(), dY.cuda())
+    torch.cuda.synchronize()
+    assert int(step.dev_status.item()) == 0
+    kw = dict(rht_block=16, grid=grid, scale_fmt=oracle.SCALE_E4M3_TENSOR, seed_rht=1)
+    sr = dict(rounding=oracle.ROUND_SR, seed_sr=2)
+    ref = {"Xr": oracle_quantize(X, oracle.AXIS_ROW, tensor_scale=ts[0], **kw), "Xc": oracle_quantize(X, oracle.AXIS_COL, tensor_scale=ts[0], **kw),
+           "Wr": oracle_quantize(W, oracle.AXIS_ROW, tensor_scale=ts[1], **kw), "Wc": oracle_quantize(W, oracle.AXIS_COL, tensor_scale=ts[1], **kw),
+           "Gr": oracle_quantize(dY, oracle.AXIS_ROW, tensor_scale=ts[2], **kw, **sr),
+           "Gc": oracle_quantize(dY, oracle.AXIS_COL, tensor_scale=ts[2], **kw, **sr)}
+    for key in ref:
+        assert_qtensor_equal(getattr(step, key), ref[key], f"{key} grid {grid}")
+    assert ufp4.gemm_path_name(step.Xr, step.Wr) == "nvf4"
+    for out, a, b, name in ((Y, "Xr", "Wr", "fwd_y"), (dX, "Gr", "Wc", "bwd_dx"), (dW, "Gc", "Xc", "bwd_dw")):
+        c, s = oracle.gemm(ref[a], ref[b])
+        assert_gemm_close(out.cpu().numpy(), c, s, f"{name} grid {grid}")
