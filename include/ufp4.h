@@ -331,6 +331,17 @@ int ufp4_debug_wait_injection(uint32_t poll_limit, int skip_loads);
  */
 int ufp4_probe_issue_rates(void *dev_scratch, size_t scratch_bytes, double *host_cycles, void *stream);
 
+/*
+ * Measurement aid (not on the hot path): cycles one SM needs to decode one pipeline stage of packed nibbles in shared
+ * memory (a CTA pair's share of a 256 x 256 x 128 step: 256 rows x 128 elements = 32768 elements) into the swizzled
+ * E5M2 operand tiles of the folded tensor-core path, with that path's decode arithmetic, when the stage is shared by
+ *   [0] 128   [1] 256   [2] 512   [3] 1024
+ * threads of one CTA per SM (host_cycles: HOST, 4 doubles).  The product kernel consumes such a stage every ~890 cycles;
+ * this is the measurement behind keeping the decode a pass of its own.  dev_scratch as for ufp4_probe_issue_rates.
+ * Synchronizes the stream.
+ */
+int ufp4_probe_decode_rate(void *dev_scratch, size_t scratch_bytes, double *host_cycles, void *stream);
+
 /* Size in bytes of the fixed scratch array behind ufp4_gemm_noalloc. */
 size_t ufp4_gemm_noalloc_max_scratch_bytes(void);
 

@@ -28,7 +28,7 @@ EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_rht
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
            "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes",
            "ufp4_diagnose_ratios", "ufp4_debug_wait_injection", "ufp4_gemm_quantized",
-           "ufp4_probe_issue_rates"]
+           "ufp4_probe_issue_rates", "ufp4_probe_decode_rate"]
 
 
 class _QTensorStruct(C.Structure):
@@ -86,6 +86,8 @@ def lib():
         L.ufp4_gemm_quantized.argtypes = [qp, qp, vp, i64, i32, u64, qp, qp, vp, sz, vp, vp]
         L.ufp4_probe_issue_rates.restype = i32
         L.ufp4_probe_issue_rates.argtypes = [vp, sz, C.POINTER(C.c_double), vp]
+        L.ufp4_probe_decode_rate.restype = i32
+        L.ufp4_probe_decode_rate.argtypes = [vp, sz, C.POINTER(C.c_double), vp]
         L.ufp4_debug_wait_injection.restype = i32
         L.ufp4_debug_wait_injection.argtypes = [C.c_uint32, i32]
         L.ufp4_diagnose_ratios.restype = i32
@@ -258,6 +260,16 @@ def probe_issue_rates(stream=None) -> dict:
     names = ["add.f32x2", "add.f32, add.f32", "lop3", "mad.lo", "add.f32x2, lop3", "add.f32x2, mad.lo",
              "add.f32x2, lop3, lop3", "add.f32, add.f32, lop3"]
     return {n: float(v) for n, v in zip(names, out)}
+
+
+def probe_decode_rate(stream=None) -> dict:
+    """ufp4_probe_decode_rate: cycles per 32768-element stage decoded in shared memory by 128 / 256 / 512 / 1024 threads of
+    one CTA per SM, and the elements per cycle that makes (see include/ufp4.h)."""
+    scratch = torch.empty(256 * 4096 + 256, dtype=torch.uint8, device="cuda")
+    out = (C.c_double * 4)()
+    _check(lib().ufp4_probe_decode_rate(scratch.data_ptr(), scratch.numel(), out, _stream_ptr(stream)))
+    return {f"{t}_threads": {"cycles_per_stage": float(v), "elements_per_cycle": 32768.0 / float(v)}
+            for t, v in zip((128, 256, 512, 1024), out)}
 
 
 def debug_wait_injection(poll_limit: int = 0, skip_loads: bool = False):
