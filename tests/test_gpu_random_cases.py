@@ -124,3 +124,51 @@ def test_grouped_gemm_random_cases(seed):
             what = f"reduction-grouped sizes {sizes} F {F16} H {Hn} fmt {fmt} path {path}"
             assert int(status.item()) == 0, what
             assert_gemm_close(got.cpu().numpy(), ref, S, what)
+
+
+def hardware_scaled_case(rng):
+    """One random product for the paths on which the tensor core applies the block scales: MX (power-of-two scales per 16
+    or per 32 elements) or NVF4 and FP16 (E4M3 block scales x a tensor scale), mixed grids, ragged shapes."""
+    fmt = int(rng.choice([oracle.SCALE_POW2, oracle.SCALE_E8M0_B32, oracle.SCALE_E4M3_TENSOR]))
+    unit = 32 if fmt == oracle.SCALE_E8M0_B32 else 16
+    M, N, K = int(rng.integers(1, 600)), int(rng.integers(1, 600)), unit * int(rng.integers(1, 1280 // unit))
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    b = rng.standard_normal((N, K)).astype(np.float32)
+    mode = int(rng.integers(0, 3))
+    if mode == 1:                         # block scales spread over 2^+-6 (inside MX's 2^14 window between neighbours), row scales beyond
+        a *= np.exp2(rng.integers(-6, 7, size=(M, K // 16)).repeat(16, 1)).astype(np.float32)
+        b *= np.exp2(rng.integers(-20, 20, size=(N, 1))).astype(np.float32)
+    elif mode == 2:
+        a[rng.random((M, K)) < 0.8] = 0
+    ga, gb = int(rng.integers(0, 3)), int(rng.integers(0, 3))
+    gmax = {oracle.GRID_INT4: 7.0, oracle.GRID_E1M2: 1.75, oracle.GRID_E2M1: 6.0}
+    kwa, kwb = {}, {}
+    if fmt == oracle.SCALE_E4M3_TENSOR:
+        kwa["tensor_scale"] = float(np.float32(4 * max(np.abs(a).max(), 1e-30) / (gmax[ga] * 448)))
+        kwb["tensor_scale"] = float(np.float32(4 * max(np.abs(b).max(), 1e-30) / (gmax[gb] * 448)))
+    A = oracle_quantize(_bf16(a), oracle.AXIS_ROW, rht_block=16, grid=ga, scale_fmt=fmt, seed_rht=3, **kwa)
+    B = oracle_quantize(_bf16(b), oracle.AXIS_ROW, rht_block=16, grid=gb, scale_fmt=fmt, seed_rht=3, **kwb)
+    paths = [ufp4.PATH_NVF4, ufp4.PATH_FP16, ufp4.PATH_AUTO] if fmt == oracle.SCALE_E4M3_TENSOR else [ufp4.PATH_MX, ufp4.PATH_TENSOR]
+    return A, B, paths, f"M {M} N {N} K {K} fmt {fmt} grids {ga},{gb} mode {mode}"
+
+
+def check_hardware_scaled_case(rng):
+    A, B, paths, what = hardware_scaled_case(rng)
+    ref, S = oracle.gemm(A, B)
+    for path in paths:
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        bf = bool(rng.integers(0, 2)) and B.rows % 8 == 0
+        out = ufp4.gemm(to_device(A), to_device(B), path=path, dev_status=status, out_bf16=bf)
+        torch.cuda.synchronize()
+        # the folded path may flag a row whose blocks spread beyond its window; the hardware-scaled paths never do here
+        if path != ufp4.PATH_TENSOR:
+            assert int(status.item()) == 0, f"{what} path {path}"
+        if int(status.item()) == 0:
+            assert_gemm_close(out.float().cpu().numpy(), ref, S, f"{what} path {path} bf16 {bf}", bf16_out=bf)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_hardware_scaled_gemm_random_cases(seed):
+    rng = np.random.default_rng(4000 + seed)
+    for _ in range(8):
+        check_hardware_scaled_case(rng)
