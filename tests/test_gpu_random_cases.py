@@ -160,9 +160,11 @@ def check_hardware_scaled_case(rng):
         bf = bool(rng.integers(0, 2)) and B.rows % 8 == 0
         out = ufp4.gemm(to_device(A), to_device(B), path=path, dev_status=status, out_bf16=bf)
         torch.cuda.synchronize()
-        # the folded path may flag a row whose blocks spread beyond its window; the hardware-scaled paths never do here
-        if path != ufp4.PATH_TENSOR:
-            assert int(status.item()) == 0, f"{what} path {path}"
+        # a flag is possible where exponents are folded into the elements: on the folded path (a row's window) and on MX with
+        # 1 x 16 scales (a block 2^14 below the other half of its 32-group, e.g. a lone tiny element among zeros); never with
+        # one hardware scale per block (E8M0 per 32, E4M3 per 16).  A flagged product is reported, not compared.
+        may_flag = path == ufp4.PATH_TENSOR or (path == ufp4.PATH_MX and A.scale_fmt == oracle.SCALE_POW2)
+        assert int(status.item()) in ((0, ufp4.DEV_EXP_WINDOW) if may_flag else (0,)), f"{what} path {path}"
         if int(status.item()) == 0:
             assert_gemm_close(out.float().cpu().numpy(), ref, S, f"{what} path {path} bf16 {bf}", bf16_out=bf)
 
