@@ -137,3 +137,38 @@ def test_diagnose_ratios_is_host_arithmetic_and_matches_the_oracle(lib):
     zero = ufp4.diagnose_ratios([0.0] * 19)
     assert np.isnan(zero[0]) and np.isnan(zero[1]) and zero[2] == pytest.approx(1.0 / 8.0)
     assert lib.ufp4_diagnose_ratios(None, None) == -1
+
+
+def test_path_selection_and_workspace_sizes_are_host_decisions(lib):
+    """ufp4_gemm_path_taken and ufp4_gemm_workspace_bytes read the operand descriptions only: which path each scale format
+    takes by default, which requests are refused, and that the workspace of a path matches what that path lays out."""
+    AUTO, EXACT, TENSOR, PROMOTE, SPLIT, FP16, MX, NVF4 = range(8)
+    taken, ws = lib.ufp4_gemm_path_taken, lib.ufp4_gemm_workspace_bytes
+    ws.restype = C.c_size_t
+
+    def q(fmt, grid=0, rows=256, k=512):
+        t = _q(rows, k, grid=grid, fmt=fmt)
+        if fmt == 2:
+            t.tensor_scale = 0x3000            # E4M3 x tensor scale: any non-null device address will do for a host decision
+        return t
+    n = C.c_int(0)
+    for fmt, want, launches in ((0, SPLIT, 2), (1, TENSOR, 2), (3, TENSOR, 2), (2, NVF4, 2)):
+        a, b = q(fmt), q(fmt, rows=128)
+        assert taken(C.byref(a), C.byref(b), AUTO, C.byref(n)) == want and n.value == launches
+        assert ws(C.byref(a), C.byref(b), AUTO) >= ws(C.byref(a), C.byref(b), want) > 0
+    assert taken(C.byref(q(1)), C.byref(q(1)), EXACT, C.byref(n)) == EXACT and n.value == 1
+    # on-request paths and the formats they refuse
+    assert taken(C.byref(q(1)), C.byref(q(3)), MX, None) == MX and taken(C.byref(q(0)), C.byref(q(1)), MX, None) == -5
+    assert taken(C.byref(q(2)), C.byref(q(2)), FP16, None) == FP16 and taken(C.byref(q(1)), C.byref(q(1)), FP16, None) == -5
+    assert taken(C.byref(q(2)), C.byref(q(1)), NVF4, None) == -5 and taken(C.byref(q(0)), C.byref(q(0)), TENSOR, None) == -5
+    assert taken(C.byref(q(1)), C.byref(q(1)), 8, None) == -4
+    assert taken(C.byref(q(1)), C.byref(q(1, k=256)), AUTO, None) == -2
+    # MX: one operand byte per element plus one 512-byte scale unit per (128 rows padded to 256, 128 elements of K)
+    a, b = q(1, rows=300, k=512), q(1, rows=128, k=512)
+    assert ws(C.byref(a), C.byref(b), MX) == 300 * 512 + 128 * 512 + (4 + 2) * 4 * 512
+    # NVF4: two half-byte planes per uniform operand, none for an E2M1 tensor, plus one scale unit per 64 elements of K
+    au, be = q(2, grid=0, rows=256, k=512), q(2, grid=2, rows=256, k=512)
+    units = 2 * 2 * 4 * 512                     # per operand: 2 stages of K x 2 row tiles x 4 steps
+    assert ws(C.byref(au), C.byref(au), NVF4) == 4 * 256 * 256 + 2 * units
+    assert ws(C.byref(be), C.byref(be), NVF4) == 2 * units
+    assert ws(C.byref(au), C.byref(be), NVF4) == 2 * 256 * 256 + 2 * units
