@@ -80,6 +80,9 @@ constexpr int kDecodeThreads = 256;
 // spread over more threads so that the grid has many more warps than the GPU has slots (no idle tail).
 template <int TPR, bool OWN>
 __global__ void __launch_bounds__(kDecodeThreads) decode_rows_kernel(const DecodeParams P) {
+    // the product kernel of the same call is launched as a programmatic dependent: its CTAs may take the SMs this grid's
+    // last wave leaves free and set themselves up; they read nothing of this grid's output before griddepcontrol.wait
+    asm volatile("griddepcontrol.launch_dependents;");
     constexpr int kRowsPerCta = kDecodeThreads / TPR;
     if ((int64_t)blockIdx.x == P.tbl_cta) {
         if (threadIdx.x == 0) {
@@ -266,6 +269,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (CG == 2) cluster_sync_all();                   // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above is independent of the decode pass; its output (operand bytes, row references, tile list) is complete
+    // and visible from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         if (lane == 0) {
@@ -660,21 +666,23 @@ int gemm_tensor_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, in
     }, &dev);
     if (rc_setup != UFP4_OK) return rc_setup;
     const int num_sms = dev->num_sms, max_pairs = dev->max_pairs;
-    if (cg == 1) {
-        const int grid = (int)(total < num_sms ? total : num_sms);
-        gemm_tc_kernel<1><<<grid, kTcThreads, kTcSmem, st>>>(tmA, tmB, tmC, P);
-        return cudaGetLastError() == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
-    }
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.gridDim = dim3(2 * (unsigned)(total < max_pairs ? total : max_pairs));
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // dependent of the decode launch above
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
     cfg.blockDim = dim3(kTcThreads);
     cfg.dynamicSmemBytes = kTcSmem;
     cfg.stream = st;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    if (cg == 1) {
+        cfg.gridDim = dim3((unsigned)(total < num_sms ? total : num_sms));
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<1>, tmA, tmB, tmC, P) == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
+    }
+    cfg.gridDim = dim3(2 * (unsigned)(total < max_pairs ? total : max_pairs));
+    cfg.numAttrs = 2;
     cudaError_t err;
     if (qmode == 1) err = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 1>, tmA, tmB, tmC, P);
     else if (qmode == 2) err = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 2>, tmA, tmB, tmC, P);
