@@ -71,6 +71,8 @@ struct MxDecodeParams {
 
 // One thread per (row, 32-group): 8 threads cover a K step, 32 threads a 512-element stretch of a row.
 __global__ void __launch_bounds__(256) decode_mx_kernel(const MxDecodeParams P) {
+    // the product kernel of the same call is a programmatic dependent launch: see its griddepcontrol.wait
+    asm volatile("griddepcontrol.launch_dependents;");
     const bool is_b = (int64_t)blockIdx.x >= P.a_ctas;
     const MxOperand &O = P.op[is_b ? 1 : 0];
     const int64_t ngroups = P.ksteps * 4;                                  // 32-groups per row, K padded to 128
@@ -199,6 +201,8 @@ gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     cluster_sync_all();                                  // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // the set-up above overlapped the decode pass's last wave; its output is complete and visible from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t t_sfa = tmem_base + kTN, t_sfb = tmem_base + kTN + 4;     // accumulator: columns 0..255, then the scales
 
     if (warp == 0) {
@@ -425,15 +429,17 @@ int gemm_mx_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, int64_
     }, &dev);
     if (rc_setup != UFP4_OK) return rc_setup;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // dependent of the decode launch above
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.gridDim = dim3(2 * (unsigned)(total < dev->max_pairs ? total : dev->max_pairs));
     cfg.blockDim = dim3(kMxThreads);
     cfg.dynamicSmemBytes = kMxSmem;
     cfg.stream = st;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, gemm_mx_kernel, tmA, tmB, tmSfA, tmSfB, tmC, P, X) == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 

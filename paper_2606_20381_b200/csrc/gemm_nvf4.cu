@@ -95,6 +95,8 @@ __device__ __forceinline__ void split_uniform8(uint32_t w, bool int4, uint32_t *
 
 // One thread per (row, 64-element MMA step): 32 bytes of codes -> 32 + 32 bytes of planes, 4 scale bytes -> one word of a unit.
 __global__ void __launch_bounds__(256) decode_nvf4_kernel(const NvDecodeParams P) {
+    // the product kernel of the same call is a programmatic dependent launch: see its griddepcontrol.wait
+    asm volatile("griddepcontrol.launch_dependents;");
     const int64_t gid0 = (int64_t)blockIdx.x * 256 + threadIdx.x;
     const bool is_b = gid0 >= P.a_threads;
     const NvOperand &O = P.op[is_b ? 1 : 0];
@@ -245,6 +247,8 @@ gemm_nvf4_kernel(const __grid_constant__ NvMaps M, const TcParams P, const NvArg
     cluster_sync_all();                                  // the peer's barriers exist before anything is signalled on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // the set-up above overlapped the decode pass's last wave; its output is complete and visible from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t t_sfa = tmem_base + kTN, t_sfb = tmem_base + kTN + 16;    // accumulator: columns 0..255, then the scales
 
     if (warp == 0) {
@@ -420,15 +424,17 @@ static int nv_launch(const NvMaps &maps, const TcParams &P, const NvArgs &X, int
     }, &dev);
     if (rc_setup != UFP4_OK) return rc_setup;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // dependent of the decode launch above
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.gridDim = dim3(2 * (unsigned)(total < dev->max_pairs ? total : dev->max_pairs));
     cfg.blockDim = dim3(kNvThreads);
     cfg.dynamicSmemBytes = Cfg::kSmem;
     cfg.stream = st;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, gemm_nvf4_kernel<PA, PB>, maps, P, X) == cudaSuccess ? UFP4_OK : UFP4_ERR_CUDA;
 }
 
