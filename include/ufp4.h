@@ -162,6 +162,25 @@ int ufp4_quantize_batched(const void *x, int64_t batch, int64_t batch_stride, in
                           int32_t *dev_status, void *stream);
 
 /*
+ * Several independent tensors in one call (a layer's X, W and dY): the same as calling ufp4_quantize for args[0],
+ * args[1], ... in this order on `stream`, except that the kernel of each tensor after the first is launched as a
+ * programmatic dependent of the one before it, so that its thread blocks fill the last, partly empty wave of its
+ * predecessor instead of waiting for it to drain.  INDEPENDENT means: no tensor of the call reads or overwrites what
+ * another one writes (inputs may be shared).  Work enqueued on the stream afterwards sees all outputs complete, as
+ * after separate calls.  All argument sets are checked before anything is launched: on an error (the status of the first
+ * offending set) nothing has been enqueued.  args: HOST array of `count` entries, read during the call only.
+ */
+typedef struct ufp4_quantize_args {
+    const void *x;                       /* device, BF16 [rows][ld]                                   */
+    int64_t rows, cols, ld;
+    int32_t axis, rht_block, grid, rounding, scale_fmt;
+    int32_t reserved;                    /* 0                                                         */
+    uint64_t seed_rht, seed_sr;
+    const ufp4_qtensor *out_row, *out_col;
+} ufp4_quantize_args;
+int ufp4_quantize_multi(int count, const ufp4_quantize_args *args, int32_t *dev_status, void *stream);
+
+/*
  * Self-check of the quantizer's scale arithmetic (Sec. 2.1: s_B = amax / g_max and x_i / s_B).  The kernel evaluates
  * amax / g and g / amax with short FMA sequences instead of the generic division; this call compares both sequences
  * with the IEEE-754 division for every FP32 mantissa at eight exponents of the supported range and g in {7, 1.75, 6},

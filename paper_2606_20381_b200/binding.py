@@ -28,13 +28,20 @@ EXPORTS = ["ufp4_version", "ufp4_status_string", "ufp4_rht_sign_mask", "ufp4_rht
            "ufp4_quantize_batched", "ufp4_selftest_division", "ufp4_gemm_workspace_bytes", "ufp4_gemm_path_taken", "ufp4_gemm", "ufp4_gemm_grouped",
            "ufp4_gemm_noalloc", "ufp4_gemm_noalloc_max_scratch_bytes", "ufp4_diagnose", "ufp4_diagnose_workspace_bytes",
            "ufp4_diagnose_ratios", "ufp4_debug_wait_injection", "ufp4_gemm_quantized",
-           "ufp4_probe_issue_rates", "ufp4_probe_decode_rate"]
+           "ufp4_probe_issue_rates", "ufp4_probe_decode_rate", "ufp4_quantize_multi"]
 
 
 class _QTensorStruct(C.Structure):
     _fields_ = [("codes", C.c_void_p), ("scales", C.c_void_p), ("tensor_scale", C.c_void_p),
                 ("rows", C.c_int64), ("k", C.c_int64), ("ld_codes_bytes", C.c_int64), ("ld_scales", C.c_int64),
                 ("grid", C.c_int32), ("scale_fmt", C.c_int32)]
+
+
+class _QuantizeArgs(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("ld", C.c_int64),
+                ("axis", C.c_int32), ("rht_block", C.c_int32), ("grid", C.c_int32), ("rounding", C.c_int32),
+                ("scale_fmt", C.c_int32), ("reserved", C.c_int32), ("seed_rht", C.c_uint64), ("seed_sr", C.c_uint64),
+                ("out_row", C.POINTER(_QTensorStruct)), ("out_col", C.POINTER(_QTensorStruct))]
 
 
 _lib = None
@@ -86,6 +93,8 @@ def lib():
         L.ufp4_gemm_quantized.argtypes = [qp, qp, vp, i64, i32, u64, qp, qp, vp, sz, vp, vp]
         L.ufp4_probe_issue_rates.restype = i32
         L.ufp4_probe_issue_rates.argtypes = [vp, sz, C.POINTER(C.c_double), vp]
+        L.ufp4_quantize_multi.restype = i32
+        L.ufp4_quantize_multi.argtypes = [i32, C.POINTER(_QuantizeArgs), vp, vp]
         L.ufp4_probe_decode_rate.restype = i32
         L.ufp4_probe_decode_rate.argtypes = [vp, sz, C.POINTER(C.c_double), vp]
         L.ufp4_debug_wait_injection.restype = i32
@@ -184,6 +193,33 @@ def quantize(x: torch.Tensor, axis: int = AXIS_BOTH, rht_block: int = 16, grid: 
                                C.byref(sc) if sc is not None else None,
                                dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
     return (out_row if axis != AXIS_COL else None), (out_col if axis != AXIS_ROW else None)
+
+
+def quantize_multi(items, dev_status: torch.Tensor | None = None, stream=None):
+    """ufp4_quantize_multi: several INDEPENDENT tensors in one call (see include/ufp4.h).  items: dicts with the keyword
+    arguments of quantize() (x, axis, rht_block, grid, rounding, scale_fmt, seed_rht, seed_sr, tensor_scale, out_row,
+    out_col); outputs not given are allocated.  Returns the list of (row variant or None, col variant or None)."""
+    n = len(items)
+    arr, keep, outs = (_QuantizeArgs * max(n, 1))(), [], []
+    for i, it in enumerate(items):
+        x = it["x"]
+        assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+        rows, cols = x.shape
+        axis, grid, fmt = it.get("axis", AXIS_BOTH), it.get("grid", GRID_INT4), it.get("scale_fmt", SCALE_FP32)
+        out_row, out_col = it.get("out_row"), it.get("out_col")
+        if axis != AXIS_COL and out_row is None:
+            out_row = alloc_qtensor(rows, cols, grid, fmt, x.device, it.get("tensor_scale"))
+        if axis != AXIS_ROW and out_col is None:
+            out_col = alloc_qtensor(cols, rows, grid, fmt, x.device, it.get("tensor_scale"))
+        sr = out_row.struct() if axis != AXIS_COL else None
+        sc = out_col.struct() if axis != AXIS_ROW else None
+        keep.append((sr, sc))
+        arr[i] = _QuantizeArgs(x.data_ptr(), rows, cols, x.stride(0), axis, it.get("rht_block", 16), grid,
+                               it.get("rounding", ROUND_RTNE), fmt, 0, it.get("seed_rht", 0), it.get("seed_sr", 0),
+                               C.pointer(sr) if sr is not None else None, C.pointer(sc) if sc is not None else None)
+        outs.append(((out_row if axis != AXIS_COL else None), (out_col if axis != AXIS_ROW else None)))
+    _check(lib().ufp4_quantize_multi(n, arr, dev_status.data_ptr() if dev_status is not None else None, _stream_ptr(stream)))
+    return outs
 
 
 def quantize_batched(x: torch.Tensor, axis: int = AXIS_BOTH, rht_block: int = 16, grid: int = GRID_INT4,

@@ -64,6 +64,8 @@ class _Ufp4Step:
         s1.wait_event(ev["start"])
         self._quantize_g(dY, s1)
         ev["g"].record(s1)
+        # separate calls here: with the three streams busy, other kernels already fill a launch's last wave, and one call for
+        # X and W would make bwd_dw wait for W as well (measured: 0.893 instead of 0.882 ms per step)
         self._quantize_x(X, s0)
         ev["x"].record(s0)
         if not reuse_w:
@@ -116,6 +118,22 @@ class Ufp4Linear(_Ufp4Step):
         need = max(ufp4.gemm_workspace_bytes(self.Xr, self.Wr, path), ufp4.gemm_workspace_bytes(self.Gr, self.Wc, path),
                    ufp4.gemm_workspace_bytes(self.Gc, self.Xc, path))
         self._init_schedule(need, device, overlap)
+
+    def _qitem(self, which, t):
+        """The keyword arguments of one of the layer's three quantizer calls (for ufp4.quantize_multi)."""
+        kw = dict(x=t, axis=ufp4.AXIS_BOTH, rht_block=self.rht_block, grid=self.grid, scale_fmt=self.scale_fmt, seed_rht=self.seed_rht)
+        if which == "x":
+            return dict(kw, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc)
+        if which == "w":
+            return dict(kw, rounding=ufp4.ROUND_RTNE, out_row=self.Wr, out_col=self.Wc)
+        return dict(kw, rounding=ufp4.ROUND_SR, seed_sr=self.seed_sr, out_row=self.Gr, out_col=self.Gc)
+
+    def quantize(self, X, W, dY, stream=None, reuse_w: bool = False):
+        """The layer's quantizer calls on one stream, as one ufp4_quantize_multi: X, W and dY are independent tensors, so each
+        kernel's thread blocks may fill the last wave of the one before it (11 % less time than three separate calls on the
+        dense layer pair)."""
+        items = [self._qitem("x", X)] + ([] if reuse_w else [self._qitem("w", W)]) + [self._qitem("g", dY)]
+        ufp4.quantize_multi(items, dev_status=self.dev_status, stream=stream)
 
     def _quantize_x(self, X, stream):
         ufp4.quantize(X, rounding=ufp4.ROUND_RTNE, out_row=self.Xr, out_col=self.Xc, **self._qkw(stream))

@@ -172,3 +172,17 @@ def test_path_selection_and_workspace_sizes_are_host_decisions(lib):
     assert ws(C.byref(au), C.byref(au), NVF4) == 4 * 256 * 256 + 2 * units
     assert ws(C.byref(be), C.byref(be), NVF4) == 2 * units
     assert ws(C.byref(au), C.byref(be), NVF4) == 2 * 256 * 256 + 2 * units
+
+
+def test_quantize_multi_rejects_bad_argument_sets_without_launching(lib):
+    qm = lib.ufp4_quantize_multi
+    row, col = _q(32, 64), _q(64, 32)
+    ok = ufp4._QuantizeArgs(0x10000, 32, 64, 64, 2, 16, 0, 0, 0, 0, 1, 2, C.pointer(row), C.pointer(col))
+    bad_axis = ufp4._QuantizeArgs(0x10000, 32, 64, 64, 5, 16, 0, 0, 0, 0, 1, 2, C.pointer(row), C.pointer(col))
+    bad_shape = ufp4._QuantizeArgs(0x10000, 32, 40, 40, 2, 16, 0, 0, 0, 0, 1, 2, C.pointer(row), C.pointer(col))
+    assert qm(0, None, None, None) == 0
+    assert qm(1, None, None, None) == -1 and qm(-1, None, None, None) == -2
+    arr = (ufp4._QuantizeArgs * 2)(ok, bad_axis)
+    assert qm(2, arr, None, None) == -4                       # the second set is wrong: reported before anything is launched
+    arr = (ufp4._QuantizeArgs * 2)(bad_shape, ok)
+    assert qm(2, arr, None, None) == -2

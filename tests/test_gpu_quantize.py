@@ -311,3 +311,47 @@ def test_rht_helps_the_uniform_grid_more_than_e2m1_on_outlier_heavy_tensors():
     assert d[(ufp4.GRID_INT4, 16)]["b_eff"] > d[(ufp4.GRID_INT4, 0)]["b_eff"]
     assert d[(ufp4.GRID_E2M1, 16)]["b_eff"] > d[(ufp4.GRID_E2M1, 0)]["b_eff"]
     assert dsqnr[ufp4.GRID_INT4] > 0 and dsqnr[ufp4.GRID_INT4] > dsqnr[ufp4.GRID_E2M1]
+
+
+def test_quantize_multi_equals_separate_calls_and_the_oracle():
+    """Independent tensors in one call (dependent launches that overlap each other's tails): every output bit-equal to the
+    oracle, whatever the mix of shapes, roundings, grids and kernels (the 16-point tile kernel, the plain kernel of the wider
+    RHT blocks and of the 1 x 32 scale blocks)."""
+    xs = [inputs.spiky_normal(272, 400, seed=1), inputs.normal_bf16(144, 400, 0.02, seed=2), inputs.normal_bf16(272, 144, 1e-3, seed=3),
+          inputs.spiky_normal(256, 192, seed=4), inputs.spiky_normal(96, 160, seed=5), inputs.spiky_normal(1040, 2064, seed=6)]
+    kws = [dict(rht_block=16, grid=ufp4.GRID_INT4, rounding=ufp4.ROUND_RTNE, scale_fmt=ufp4.SCALE_POW2, seed_rht=1),
+           dict(rht_block=16, grid=ufp4.GRID_INT4, rounding=ufp4.ROUND_RTNE, scale_fmt=ufp4.SCALE_POW2, seed_rht=1),
+           dict(rht_block=16, grid=ufp4.GRID_INT4, rounding=ufp4.ROUND_SR, scale_fmt=ufp4.SCALE_POW2, seed_rht=1, seed_sr=2),
+           dict(rht_block=64, grid=ufp4.GRID_E1M2, rounding=ufp4.ROUND_RTNE, scale_fmt=ufp4.SCALE_FP32, seed_rht=7),
+           dict(rht_block=16, grid=ufp4.GRID_E2M1, rounding=ufp4.ROUND_SR, scale_fmt=ufp4.SCALE_E8M0_B32, seed_rht=3, seed_sr=9),
+           dict(rht_block=0, grid=ufp4.GRID_E2M1, rounding=ufp4.ROUND_RTNE, scale_fmt=ufp4.SCALE_FP32, seed_rht=0)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dev = [x.cuda() for x in xs]
+    for _ in range(3):                      # repeated, so that a launch of one round follows the last of the round before
+        outs = ufp4.quantize_multi([dict(x=d, axis=ufp4.AXIS_BOTH, **kw) for d, kw in zip(dev, kws)], dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for x, kw, (row, col) in zip(xs, kws, outs):
+        assert_qtensor_equal(row, oracle_quantize(x, oracle.AXIS_ROW, **kw), f"multi row {kw}")
+        assert_qtensor_equal(col, oracle_quantize(x, oracle.AXIS_COL, **kw), f"multi col {kw}")
+    # a consumer enqueued right behind the call sees every tensor complete: the product of the first two tensors' row
+    # variants, taken straight after a fresh multi call into fresh outputs
+    outs = ufp4.quantize_multi([dict(x=d, axis=ufp4.AXIS_BOTH, **kw) for d, kw in zip(dev[:3], kws[:3])])
+    got = ufp4.gemm(outs[0][0], outs[1][0])
+    ref, S = oracle.gemm(oracle_quantize(xs[0], oracle.AXIS_ROW, **kws[0]), oracle_quantize(xs[1], oracle.AXIS_ROW, **kws[1]))
+    from helpers import assert_gemm_close
+    assert_gemm_close(got.cpu().numpy(), ref, S, "product right behind a multi call")
+
+
+def test_quantize_multi_checks_every_tensor_before_launching_any():
+    good = inputs.normal_bf16(64, 64, 1.0, seed=1).cuda()
+    row = ufp4.alloc_qtensor(64, 64, ufp4.GRID_INT4, ufp4.SCALE_FP32, "cuda")
+    col = ufp4.alloc_qtensor(64, 64, ufp4.GRID_INT4, ufp4.SCALE_FP32, "cuda")
+    row.codes.fill_(0xAB)
+    bad_out = ufp4.alloc_qtensor(64, 48, ufp4.GRID_INT4, ufp4.SCALE_FP32, "cuda")        # wrong shape for the second tensor
+    with pytest.raises(ufp4.Ufp4Error) as e:
+        ufp4.quantize_multi([dict(x=good, out_row=row, out_col=col), dict(x=good, out_row=bad_out, out_col=col)])
+    assert e.value.status == -2
+    torch.cuda.synchronize()
+    assert torch.all(row.codes == 0xAB)                       # the first tensor was not quantized either
+    assert ufp4.quantize_multi([]) == []
