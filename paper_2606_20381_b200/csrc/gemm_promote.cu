@@ -179,7 +179,7 @@ gemm_promote_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(pempty_bar + 8 * b, 8);
         }
         abort_flag[0] = (base & 1023u) ? 1u : 0u;
-        abort_flag[1] = kWaitLimit;
+        abort_flag[1] = P.wait_limit ? P.wait_limit : kWaitLimit;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -197,7 +197,7 @@ gemm_promote_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+            for (int tile = blockIdx.x; ok && !P.skip_loads && tile < P.total_tiles; tile += gridDim.x) {
                 const PTile t = ptile_info(P, tile);
                 for (int ks = 0; ks < t.nks; ++ks) {
                     if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -409,6 +409,8 @@ int gemm_promote_launch(const ufp4_qtensor *A, const ufp4_qtensor *B, void *C, i
     if (total < 1 || total > 0x7FFFFFFF) return UFP4_ERR_SHAPE;
     P.total_tiles = (int)total;
     P.n_unaligned = ((N * (c_is_bf16 ? 2 : 4)) % 16) != 0;
+    P.wait_limit = debug_wait_limit();
+    P.skip_loads = debug_skip_loads();
 
     static DeviceSetup slots[kMaxDevices];
     const DeviceSetup *dev = nullptr;

@@ -25,6 +25,7 @@ def _operands(M, N, K, scale_fmt):
 
 
 @pytest.mark.parametrize("path,scale_fmt", [(ufp4.PATH_TENSOR, oracle.SCALE_POW2), (ufp4.PATH_SPLIT, oracle.SCALE_FP32),
+                                            (ufp4.PATH_PROMOTE, oracle.SCALE_FP32),
                                             (ufp4.PATH_FP16, oracle.SCALE_E4M3_TENSOR), (ufp4.PATH_MX, oracle.SCALE_E8M0_B32),
                                             (ufp4.PATH_NVF4, oracle.SCALE_E4M3_TENSOR)])
 @pytest.mark.parametrize("shape", [(384, 512, 256), (4096, 4096, 256)])     # a few tiles; more tiles than CTA pairs
